@@ -15,7 +15,7 @@
  *                     Sec. 3.3.1 / App. E.2).
  *
  *   (ii) orc_emu_*  : the tiled algorithms step by step, Algorithm 1
- *                     (standard), Algorithm 3 (stabilised, the magenta lines)
+ *                     (standard), Algorithm 3 (stabilised: Algorithm 1 plus three added steps)
  *                     and Algorithm 2 (backward), in emulated FP32 with the
  *                     BF16 rounding points the paper's analysis fixes:
  *                     P-bar is a BF16 value (Sec. 4 relies on entries of P-bar
@@ -263,6 +263,25 @@ void orc_ref_delta_dp(const double *q, const double *k, const double *v, const d
 /* (ii) emulated tiled algorithms.                                      */
 /* ------------------------------------------------------------------ */
 
+/* The tie rule of Sec. 4 / Algorithm 3 for one row of one key block: given the n scaled scores of the
+ * block (masked entries are -inf), r_m = rowmax, r_s = #{r_m - s <= eps} (the maximum itself counts; for a
+ * masked entry r_m - (-inf) = inf is not counted), and the returned m' is
+ *   beta r_m if r_m > 0 and r_s > 1;   0 if r_m < 0 and r_s > 1;   r_m otherwise.
+ * This is the only copy of the rule: orc_emu_fwd calls it for every row and block, and the hand-made rows of
+ * the tests drive it both directly and through orc_emu_fwd. */
+float orc_tie_rule(const float *s, int n, float beta, float eps, int *r_s_out)
+{
+    float r_m = -INFINITY;
+    for (int t = 0; t < n; ++t) if (s[t] > r_m) r_m = s[t];
+    int r_s = 0;
+    for (int t = 0; t < n; ++t) if (r_m - s[t] <= eps) r_s += 1;
+    float mp = r_m;
+    if (r_m > 0.0f && r_s > 1) mp = beta * r_m;
+    if (r_m < 0.0f && r_s > 1) mp = 0.0f;
+    if (r_s_out) *r_s_out = r_s;
+    return mp;
+}
+
 /*
  * Forward, Algorithm 1 (mode 0) / Algorithm 3 (mode 1).
  *
@@ -328,8 +347,7 @@ void orc_emu_fwd(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                     float mp = r_m;
                     if (mode == 1) {
                         int r_s = 0;
-                        for (int t = t0; t < t1; ++t)
-                            if (r_m - s[t - t0] <= eps) r_s += 1;   /* -inf entries: r_m - (-inf) = inf, not counted */
+                        const float mp_rule = orc_tie_rule(s, t1 - t0, beta, eps, &r_s);   /* Algorithm 3's three added steps */
                         if (guard_cap > 0.0f) {
                             /* Guarded variant (an extension, not in the paper): the maximum also counts as repeated
                              * when it equals, within eps, the largest row maximum of the earlier blocks (a tie split
@@ -342,8 +360,7 @@ void orc_emu_fwd(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                             if (repeated && r_m > 0.0f) mp = ((beta - 1.0f) * r_m <= guard_cap) ? beta * r_m : r_m + guard_cap;
                             if (repeated && r_m < 0.0f) mp = (-r_m <= guard_cap) ? 0.0f : r_m + guard_cap;
                         } else {
-                            if (r_m > 0.0f && r_s > 1) mp = beta * r_m;
-                            if (r_m < 0.0f && r_s > 1) mp = 0.0f;
+                            mp = mp_rule;
                         }
                     }
                     const float m_new = (m > mp) ? m : mp;
@@ -505,21 +522,6 @@ void orc_emu_bwd(const uint16_t *q, const uint16_t *k, const uint16_t *v,
             free(dq);
         }
     }
-}
-
-/* One row of the tie rule of Sec. 4 / Algorithm 3, exposed for hand-made
- * rows: given n scores, returns m' and (through r_s_out) the count r_s. */
-float orc_tie_rule(const float *s, int n, float beta, float eps, int *r_s_out)
-{
-    float r_m = -INFINITY;
-    for (int t = 0; t < n; ++t) if (s[t] > r_m) r_m = s[t];
-    int r_s = 0;
-    for (int t = 0; t < n; ++t) if (r_m - s[t] <= eps) r_s += 1;
-    float mp = r_m;
-    if (r_m > 0.0f && r_s > 1) mp = beta * r_m;
-    if (r_m < 0.0f && r_s > 1) mp = 0.0f;
-    if (r_s_out) *r_s_out = r_s;
-    return mp;
 }
 
 /* Prefix trace of Sec. 3.3.2: for one row of BF16 weights p[0..n) and one

@@ -95,6 +95,61 @@ def test_tie_rule_rows(golden_dir):
     assert (mp, rs) == (8.0, 2)
 
 
+def _row_as_attention(scores, d=4):
+    """Inputs whose (unscaled) scores q . k_t are the given numbers, for every query row: q = (1, ..., 1) and
+    k_t = the score split into d BF16 pieces (largest first), so that the FP32 dot product adds them back
+    without rounding when the score has at most 8 d significant bits."""
+    n = len(scores)
+    k = np.zeros((1, 1, n, d), np.float32)
+    for t, sc in enumerate(scores):
+        rest = np.float64(sc)
+        for c in range(d):
+            piece = float(ai.bf16_bits_to_f32(ai.to_bf16_bits(np.array([rest], np.float32)))[0])
+            k[0, 0, t, c] = piece
+            rest -= piece
+    q = np.ones((1, 1, n, d), np.float32)
+    v = np.ones((1, 1, n, d), np.float32)
+    realised = k.astype(np.float64).sum(-1)[0, 0]
+    return ai.to_bf16_bits(q), ai.to_bf16_bits(k), ai.to_bf16_bits(v), realised
+
+
+def test_tie_rule_rows_through_the_tiled_forward(golden_dir):
+    """The same hand-made rows, and rows on the eps boundary, driven through emu_fwd itself (one key block, every
+    query row sees the row of scores): the running maximum it reports is m' of Algorithm 3, in the standard
+    mode it is r_m, and the largest P-bar is bf16(exp(r_m - m'))."""
+    def rows(name, cols):
+        for line in open(os.path.join(golden_dir, name)):
+            line = line.strip()
+            if line and not line.startswith("#"):
+                parts = [x.strip() for x in line.split(";")]
+                assert len(parts) == cols, line
+                yield parts
+    cases = [(1.0, 1e-3, sc, mp) for sc, mp, _ in rows("tie_rule_rows.txt", 3)]
+    cases += [(float(a), float(e), sc, mp) for a, e, sc, mp in rows("tie_rule_boundary_rows.txt", 4)]
+    assert len(cases) == 15
+    for alpha, eps, sc, mp in cases:
+        scores = [float(x) for x in sc.split()]
+        q, k, v, realised = _row_as_attention(scores)
+        assert np.max(np.abs(realised - np.array(scores))) <= 2e-7 * max(1.0, max(abs(x) for x in scores)), sc
+        n = len(scores)
+        r_m = np.float32(alpha) * np.float32(realised.max())
+        for mode in (0, 1):
+            _, _, dg = oracle.emu_fwd(q, k, v, False, alpha, mode, beta=2.0, eps=eps, Br=n, Bc=n, diagnostics=True)
+            want_m = np.float32(float(mp)) if mode == 1 else r_m
+            if mode == 1 and float(mp) not in (0.0, 2.0 * float(r_m)):
+                want_m = r_m                      # the rule did not fire: m' is the block maximum as realised in FP32
+            assert np.all(dg["m"] == want_m), (sc, alpha, eps, mode, dg["m"][0, 0, 0], want_m)
+            want_pmax = ai.bf16_bits_to_f32(ai.to_bf16_bits(np.array([np.exp(np.float64(r_m) - np.float64(want_m))], np.float32)))[0]
+            assert np.all(dg["pmax"] == want_pmax), (sc, mode)
+    # a wrong scale on eps or a strict comparison must change at least the four boundary rows above: check that the
+    # boundary rows really sit on the boundary (difference of the two largest scaled scores == eps exactly)
+    on_boundary = 0
+    for a, e, sc, mp in rows("tie_rule_boundary_rows.txt", 4):
+        s = sorted((np.float32(a) * np.float32(x) for x in map(float, sc.split())), reverse=True)
+        on_boundary += int(np.float32(s[0] - s[1]) == np.float32(e))
+    assert on_boundary == 4
+
+
 @pytest.fixture(scope="module")
 def c3_sample():
     t, m = ai.make("C3", B=1, H=8)
