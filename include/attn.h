@@ -42,6 +42,12 @@
  *  - Device-side waits are bounded.  If one runs out (a pipeline fault), the
  *    kernel stops early and records it; attn_last_device_status() reports it
  *    after the caller has synchronised the stream.
+ *  - Host threads: every entry point may be called from several host threads
+ *    at once, each with its own current device and stream; what the library
+ *    caches on the host is per device and published atomically.  The
+ *    parameters set by attn_set_mitigation() and attn_set_guard_max_shift()
+ *    are process-wide: a compute call uses the values in force when it is
+ *    made.  attn_bwd_static() shares one scratch array per device (see there).
  */
 #ifndef ATTN_H_
 #define ATTN_H_
@@ -310,8 +316,22 @@ int attn_get_mitigation(float* beta, float* eps);
 
 /* After the caller has synchronised `stream`: ATTN_OK, or ATTN_ERR_TIMEOUT if a
  * kernel enqueued by this library on the current device gave up on a bounded
- * wait since the last call of this function (which clears the record). */
+ * wait since the last call of this function (which clears the record), or
+ * ATTN_ERR_CUDA if a kernel found its shared-memory layout out of bounds. */
 int attn_last_device_status(void* stream);
+
+/*
+ * Self-test of the bounded-wait path (the paper has no counterpart: this belongs to the error contract of the
+ * library, not to the method).  Enqueues on `stream` a one-block kernel built like the compute kernels (barriers in
+ * shared memory, a TMEM allocation, one single-thread role and one whole-warp role, the common teardown) in which
+ * nothing ever arrives on the barriers the roles wait for.  Their waits are bounded at one millisecond instead of the
+ * compute kernels' two seconds, so the kernel gives up after about a millisecond through the path a pipeline fault
+ * would take: abort flag, every role leaves its wait, TMEM is freed, the device status word is set.  After the caller
+ * has synchronised, attn_last_device_status() returns ATTN_ERR_TIMEOUT once; the context is intact and later calls
+ * behave normally.  No fault, trap or unbounded loop is involved.  Returns ATTN_OK once enqueued, ATTN_ERR_DEVICE /
+ * ATTN_ERR_CUDA as the compute entry points.
+ */
+int attn_selftest_wait_timeout(void* stream);
 
 /* Static, human-readable text for a return code. */
 const char* attn_strerror(int code);

@@ -14,12 +14,12 @@ import os
 from . import build as _build
 
 __all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
-           "attn_get_tiles", "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status",
+           "attn_get_tiles", "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout",
            "attn_strerror", "lib", "LIB_PATH", "EXPORTS"]
 
 LIB_PATH = _build.LIB
 EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
-           "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_strerror")
+           "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout", "attn_strerror")
 
 
 class AttnError(RuntimeError):
@@ -78,6 +78,8 @@ def _load():
     L.attn_get_mitigation.argtypes = [C.POINTER(f), C.POINTER(f)]
     L.attn_last_device_status.restype = i
     L.attn_last_device_status.argtypes = [vp]
+    L.attn_selftest_wait_timeout.restype = i
+    L.attn_selftest_wait_timeout.argtypes = [vp]
     L.attn_strerror.restype = C.c_char_p
     L.attn_strerror.argtypes = [i]
     return L
@@ -229,3 +231,8 @@ def attn_get_mitigation():
 def attn_last_device_status(stream=None):
     """Call after synchronising. Returns 0 or the ATTN_ERR_TIMEOUT code (does not raise)."""
     return int(lib.attn_last_device_status(_stream(stream) if stream is not None else None))
+
+
+def attn_selftest_wait_timeout(stream=None):
+    """Enqueue the kernel whose bounded waits run out by construction (about a millisecond); see attn.h."""
+    _check(lib.attn_selftest_wait_timeout(_stream(stream) if stream is not None else None), "attn_selftest_wait_timeout")

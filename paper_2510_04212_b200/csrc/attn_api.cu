@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <atomic>
 #include <utility>
 
 #include "../../include/attn.h"
@@ -13,6 +14,7 @@
 #include "bwd_kernel_d128.cuh"
 #include "delta_dp_kernel.cuh"
 #include "fwd_kernel.cuh"
+#include "selftest_kernel.cuh"
 
 // Scratch for attn_bwd_static(): lives in the library's device image, so every GPU that loads the
 // library holds these bytes until the process exits.  In host code this name is only a handle for
@@ -21,14 +23,15 @@ static __device__ __align__(256) unsigned char g_static_bwd_scratch[ATTN_BWD_STA
 
 namespace {
 
-__device__ int g_device_status = 0;       // set to 1 by a kernel whose bounded wait ran out
+__device__ int g_device_status = 0;       // set by a kernel: 1 = a bounded wait ran out, 2 = shared-memory layout check failed
 
-#ifdef ATTN_TRACE
-unsigned long long* g_trace = nullptr;
-#endif
-float g_beta = 2.0f;
-float g_eps = 1e-3f;
-float g_guard_cap = ATTN_GUARD_DEFAULT_MAX_SHIFT;
+// Host-side state.  Entry points may be called from several host threads at once (each with its own current device
+// and stream): the process-wide parameters are atomics, everything cached per device is an array indexed by the
+// device ordinal and written once with release / read with acquire.
+constexpr int MAX_DEVICES = 64;
+std::atomic<float> g_beta{2.0f};
+std::atomic<float> g_eps{1e-3f};
+std::atomic<float> g_guard_cap{ATTN_GUARD_DEFAULT_MAX_SHIFT};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -36,16 +39,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 EncodeTiledFn get_encoder()
 {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    static std::atomic<EncodeTiledFn> fn{nullptr};
+    EncodeTiledFn f = fn.load(std::memory_order_acquire);
+    if (!f) {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
             q != cudaDriverEntryPointSuccess)
             return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
+        f = reinterpret_cast<EncodeTiledFn>(p);
+        fn.store(f, std::memory_order_release);     // two threads may both look it up: they store the same pointer
     }
-    return fn;
+    return f;
 }
 
 // [rows, d] BF16 row-major viewed as a 2D tensor; one box = box_rows rows x 64 columns (128 bytes,
@@ -87,18 +92,47 @@ int check_shape(int B, int H, int N, int d)
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Compute-capability major and SM count of the current device, looked up once per device.
+struct DeviceInfo { int major, sm_count; };
+int device_info(DeviceInfo* out, int* dev_out = nullptr)
+{
+    static std::atomic<int> packed[MAX_DEVICES];      // 0 = not looked up yet; else (major << 16) | sm_count
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return ATTN_ERR_CUDA;
+    int v = packed[dev].load(std::memory_order_acquire);
+    if (!v) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || major <= 0 || sms <= 0)
+            return ATTN_ERR_CUDA;
+        v = (major << 16) | sms;
+        packed[dev].store(v, std::memory_order_release);
+    }
+    out->major = v >> 16;
+    out->sm_count = v & 0xFFFF;
+    if (dev_out) *dev_out = dev;
+    return ATTN_OK;
+}
+
 int check_device()
 {
+    DeviceInfo di;
+    if (int e = device_info(&di)) return e;
+    return di.major == 10 ? ATTN_OK : ATTN_ERR_DEVICE;
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is per device and per kernel: set it once for each (kernel, device).
+template <auto Kern>
+int ensure_dynamic_smem(int bytes)
+{
+    static std::atomic<bool> done[MAX_DEVICES];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
-    static int cached_dev = -1, cached_major = -1;
-    if (dev != cached_dev) {
-        int major = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ATTN_ERR_CUDA;
-        cached_dev = dev;
-        cached_major = major;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return ATTN_ERR_CUDA;
+    if (!done[dev].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return ATTN_ERR_CUDA;
+        done[dev].store(true, std::memory_order_release);
     }
-    return cached_major == 10 ? ATTN_OK : ATTN_ERR_DEVICE;
+    return ATTN_OK;
 }
 
 int* status_ptr()
@@ -132,15 +166,8 @@ int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
                const attn::FwdParams& prm, cudaStream_t st)
 {
     using Cfg = attn::FwdCfg<D>;
-    auto kern = attn::attn_fwd_kernel<D, MODE, CAUSAL, COUNT, PADDED>;
-    static int configured_dev = -1;            // the attribute is per device and per kernel instantiation
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (configured_dev != dev) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        configured_dev = dev;
-    }
+    constexpr auto kern = attn::attn_fwd_kernel<D, MODE, CAUSAL, COUNT, PADDED>;
+    if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
     return launch_pdl(kern, dim3(prm.Tr * prm.BH), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tq, tk, tv, to, prm) == cudaSuccess
                ? ATTN_OK : ATTN_ERR_CUDA;
 }
@@ -150,15 +177,8 @@ int launch_bwd_d128(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensor
                     const CUtensorMap& tdk, const CUtensorMap& tdv, const attn::BwdParams& prm, cudaStream_t st)
 {
     using Cfg = attn::Bwd128Cfg;
-    auto kern = attn::attn_bwd_kernel_d128<CAUSAL, GENERAL>;
-    static int configured_dev = -1;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (configured_dev != dev) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        configured_dev = dev;
-    }
+    constexpr auto kern = attn::attn_bwd_kernel_d128<CAUSAL, GENERAL>;
+    if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
     return launch_pdl(kern, dim3(prm.Tr * prm.BH), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tq, tk, tv, tdo, tdk, tdv,
                       prm) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
@@ -169,17 +189,11 @@ int launch_bwd_d64(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorM
                    const attn::BwdParams& prm, cudaStream_t st)
 {
     using Cfg = attn::Bwd64Cfg;
-    auto kern = attn::attn_bwd_kernel_d64<CAUSAL, GENERAL>;
-    static int configured_dev = -1;
-    static int sm_count = 0;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (configured_dev != dev) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            return ATTN_ERR_CUDA;
-        configured_dev = dev;
-    }
+    constexpr auto kern = attn::attn_bwd_kernel_d64<CAUSAL, GENERAL>;
+    if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
+    DeviceInfo di;
+    if (int e = device_info(&di)) return e;
+    const int sm_count = di.sm_count;
     // persistent: one CTA per SM walks the (head, key tile) items
     const long long items = static_cast<long long>(prm.Tr) * prm.BH;
     const unsigned grid = static_cast<unsigned>(items < sm_count ? items : sm_count);
@@ -213,15 +227,8 @@ int launch_delta_dp(const void* q, const void* k, const void* v, const void* dO,
                            int BH, int N, float scale, cudaStream_t st)
 {
     using Cfg = attn::DeltaDpCfg<D>;
-    auto kern = attn::delta_dp_kernel<D, CAUSAL>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATTN_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        configured[dev] = true;
-    }
+    constexpr auto kern = attn::delta_dp_kernel<D, CAUSAL>;
+    if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
     kern<<<static_cast<unsigned>((N / Cfg::ROWS) * BH), 256, Cfg::SMEM_BYTES, st>>>(
         static_cast<const uint4*>(q), static_cast<const uint4*>(k), static_cast<const uint4*>(v),
         static_cast<const uint4*>(dO), lse, delta, N, scale);
@@ -231,10 +238,6 @@ int launch_delta_dp(const void* q, const void* k, const void* v, const void* dO,
 }  // namespace
 
 extern "C" {
-
-#ifdef ATTN_TRACE
-void attn_debug_set_trace(unsigned long long* p) { g_trace = p; }
-#endif
 
 // attn_fwd and attn_fwd_count_ones: `ones` == nullptr selects the instantiations without the counter
 static int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int* ones,
@@ -263,9 +266,6 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
         return ATTN_ERR_CUDA;
 
     attn::FwdParams prm;
-#ifdef ATTN_TRACE
-    prm.trace = g_trace;
-#endif
     prm.lse = lse;
     prm.ones = ones;
     prm.pbar_fmt = pbar_fmt;
@@ -278,9 +278,9 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     prm.H = H;
     prm.group = H / Hkv;
     prm.scale = scale;
-    prm.beta = g_beta;
-    prm.eps = g_eps;
-    prm.guard_cap = (mode & ATTN_MODE_FLAG_GUARDED) ? g_guard_cap : 0.0f;
+    prm.beta = g_beta.load();
+    prm.eps = g_eps.load();
+    prm.guard_cap = (mode & ATTN_MODE_FLAG_GUARDED) ? g_guard_cap.load() : 0.0f;
     prm.status = status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int key = (d == 128 ? 8 : 0) | ((mode & ATTN_MODE_STABILISED) ? 4 : 0) | (causal ? 2 : 0) | (ones ? 1 : 0);
@@ -403,9 +403,6 @@ static int bwd_stage_impl(int stage, const void* q, const void* k, const void* v
             !make_map(&tdo, dO, rows, d))
             return ATTN_ERR_CUDA;
         attn::BwdParams prm;
-#ifdef ATTN_TRACE
-        prm.trace = g_trace;
-#endif
         prm.lse = lse;
         prm.delta = delta;
         prm.dq_acc = acc;
@@ -533,23 +530,24 @@ int attn_bwd_static(const void* q, const void* k, const void* v, const void* o, 
                     void* dq, void* dk, void* dv, float* delta,
                     int B, int H, int N, int d, int causal, float scale, int mode, void* stream)
 {
+    // same order of checks as attn_bwd: pointers, shape, then the scratch size
+    if (!q || !k || !v || !o || !dO || !lse || !dq || !dk || !dv || !delta) return ATTN_ERR_NULL;
     if (int e = check_shape(B, H, N, d)) return e;
     const size_t need = attn_bwd_workspace_bytes(B, H, N, d);
     if (need > static_cast<size_t>(ATTN_BWD_STATIC_MAX_BYTES)) return ATTN_ERR_WORKSPACE;   // problem too large for the built-in scratch
     if (int e = check_device()) return e;
     // Set-up, once per device, with that device current: translate the symbol into the device
     // address of this device's copy of the array.  No memory is allocated here or anywhere below.
-    constexpr int MAX_DEVICES = 64;
-    static void* scratch_addr[MAX_DEVICES] = {nullptr};
+    static std::atomic<void*> scratch_addr[MAX_DEVICES];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return ATTN_ERR_CUDA;
-    if (!scratch_addr[dev]) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_bwd_scratch) != cudaSuccess || !p) return ATTN_ERR_CUDA;
-        scratch_addr[dev] = p;
+    void* scratch = scratch_addr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        if (cudaGetSymbolAddress(&scratch, g_static_bwd_scratch) != cudaSuccess || !scratch) return ATTN_ERR_CUDA;
+        scratch_addr[dev].store(scratch, std::memory_order_release);
     }
     // Same three kernels as attn_bwd; the first one clears the part of the scratch this call uses.
-    return attn_bwd_stage(ATTN_BWD_STAGE_ALL, q, k, v, o, dO, lse, dq, dk, dv, delta, scratch_addr[dev],
+    return attn_bwd_stage(ATTN_BWD_STAGE_ALL, q, k, v, o, dO, lse, dq, dk, dv, delta, scratch,
                           static_cast<size_t>(ATTN_BWD_STATIC_MAX_BYTES), B, H, N, d, causal, scale, mode, stream);
 }
 
@@ -565,25 +563,25 @@ int attn_get_tiles(int d, int* Br, int* Bc)
 int attn_set_guard_max_shift(float max_shift)
 {
     if (!(max_shift > 0.0f) || !isfinite(max_shift)) return ATTN_ERR_PARAM;
-    g_guard_cap = max_shift;
+    g_guard_cap.store(max_shift);
     return ATTN_OK;
 }
 
-float attn_get_guard_max_shift(void) { return g_guard_cap; }
+float attn_get_guard_max_shift(void) { return g_guard_cap.load(); }
 
 int attn_set_mitigation(float beta, float eps)
 {
     if (!(beta > 1.0f) || !isfinite(beta) || !(eps > 0.0f) || !isfinite(eps)) return ATTN_ERR_PARAM;
-    g_beta = beta;
-    g_eps = eps;
+    g_beta.store(beta);
+    g_eps.store(eps);
     return ATTN_OK;
 }
 
 int attn_get_mitigation(float* beta, float* eps)
 {
     if (!beta || !eps) return ATTN_ERR_NULL;
-    *beta = g_beta;
-    *eps = g_eps;
+    *beta = g_beta.load();
+    *eps = g_eps.load();
     return ATTN_OK;
 }
 
@@ -596,9 +594,18 @@ int attn_last_device_status(void* stream)
     if (flag) {
         const int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return ATTN_ERR_CUDA;
-        return ATTN_ERR_TIMEOUT;
+        return flag == 1 ? ATTN_ERR_TIMEOUT : ATTN_ERR_CUDA;     // 2: a kernel found its shared-memory layout out of bounds
     }
     return ATTN_OK;
+}
+
+int attn_selftest_wait_timeout(void* stream)
+{
+    if (int e = check_device()) return e;
+    int* status = status_ptr();
+    if (!status) return ATTN_ERR_CUDA;
+    attn::wait_timeout_selftest_kernel<1000000ull><<<1, 96, 0, static_cast<cudaStream_t>(stream)>>>(status);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 const char* attn_strerror(int code)
@@ -607,7 +614,7 @@ const char* attn_strerror(int code)
         case ATTN_OK: return "ok";
         case ATTN_ERR_NULL: return "a required pointer is NULL";
         case ATTN_ERR_SHAPE: return "unsupported shape (need d in {64,128}, N a multiple of 128, B,H >= 1)";
-        case ATTN_ERR_MODE: return "mode must be 0 (standard) or 1 (stabilised)";
+        case ATTN_ERR_MODE: return "mode holds a bit this entry point does not accept (0 or 1, plus the ATTN_MODE_FLAG_* it documents)";
         case ATTN_ERR_PARAM: return "parameter out of range (scale > 0, beta > 1, eps > 0, all finite)";
         case ATTN_ERR_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";
         case ATTN_ERR_CUDA: return "a CUDA call or kernel launch failed";

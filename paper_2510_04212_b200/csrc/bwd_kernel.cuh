@@ -10,7 +10,6 @@
 #pragma once
 #include <cuda.h>
 #include "ptx.cuh"
-#include "fwd_kernel.cuh"
 
 namespace attn {
 
@@ -95,9 +94,6 @@ dq_convert_tiled128_kernel(const float4* __restrict__ acc, uint4* __restrict__ d
 
 // ------------------------------------------------------------------ arguments of the main backward kernels
 struct BwdParams {
-#ifdef ATTN_TRACE
-    unsigned long long* trace;
-#endif
     const float* lse;
     const float* delta;
     float* dq_acc;

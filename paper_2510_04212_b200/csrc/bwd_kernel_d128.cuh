@@ -94,7 +94,6 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     int& abort_flag = *reinterpret_cast<int*>(misc + 2308);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) TRACE(0);
     // Causal: key tile 0 sees the most query tiles, so the tile 0 of several heads first (longest jobs first) -- of
     // as many heads as keep their tensors and FP32 dQ accumulators in L2 together (the host chooses the group;
     // B=2,H=16,N=8192: all 32 heads at once 1.43 ms, groups of 4 to 8 heads 1.35-1.37 ms).  Full attention: every job
@@ -339,7 +338,6 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             ok = mbar_wait(bar(VEC_FULL + buf), (it >> 1) & 1, &abort_flag) && mbar_wait(bar(S_FULL), it & 1, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (warp == 0) TRACE(16 + (it < 60 ? it : 59) * 4 + 0);
             tc_fence_after();
             // DIAG (compile time): a partly masked pair: the causal diagonal (first query tile of a query head: key row r
             // sees query column q only if r <= q), key rows or query columns beyond the sequence length.  Key row r sees the
@@ -390,12 +388,10 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(P_FULL));                             // dV(i) and S^T(i+1) run behind the second half
-            if (warp == 0) TRACE(16 + (it < 60 ? it : 59) * 4 + 2);
             // ---- second half: dS^T = P o (dP^T - delta), rounded to BF16, into shared memory for dQ and dK
             ok = mbar_wait(bar(DP_FULL), it & 1, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (warp == 0) TRACE(16 + (it < 60 ? it : 59) * 4 + 3);
             tc_fence_after();
             auto ds_phase = [&](auto diag_tag) {
                 constexpr bool DIAG = decltype(diag_tag)::value;
@@ -437,7 +433,6 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             fence_proxy_async_smem();
             tc_fence_before();
             mbar_arrive(bar(DS_FULL));
-            if (warp == 0) TRACE(16 + (it < 60 ? it : 59) * 4 + 1);
         }
         // ---- dV (warps 0-3) and scale * dK (warps 4-7) -> BF16 -> the two Q stages (free now: every MMA has completed
         // and nothing more is loaded), in the layout of a loaded tile -> TMA stores
@@ -485,11 +480,9 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     if (abort_flag) {
         for (int t = 0; t < 64; ++t) __nanosleep(1000);
     }
-    if (tid == 0) TRACE(4);
     tc_fence_before();
     __syncthreads();
     if (warp == 13) tmem_dealloc(tmem_base_s, Cfg::TMEM_COLS);
-    if (tid == 0) TRACE(5);
     if (tid == 0 && abort_flag) atomicExch(prm.status, 1);
 }
 

@@ -181,7 +181,6 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     static_assert(NBARS * 8 <= 256 && 2312 + 32 <= Cfg::MISC_BYTES, "misc layout");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) TRACE(0);
     griddep_launch_dependents();
     auto bar = [&](int b) { return smem_u32(&bars[b]); };
 
@@ -552,7 +551,6 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 ok = mbar_wait_ool(bar(VEC_FULL + buf), (g >> 1) & 1, &abort_flag) && mbar_wait_ool(bar(SDP_FULL), g & 1, &abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (warp == 0) TRACE(16 + (g < 60 ? g : 59) * 4 + 0);
                 tc_fence_after();
                 uint8_t* xrow = sX_ptr + buf * Cfg::X_BYTES + half * Cfg::TILE_BYTES + r * 128;
                 // the pair on the causal diagonal: key row r sees query column q only if r <= q.  One copy of the arithmetic
@@ -609,12 +607,10 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             dsk[(c >> 1) + 1] = pack_bf16(ds[2], ds[3]);
                         }
                         if (h == 0) {
-                            if (warp == 0) TRACE(16 + (g < 60 ? g : 59) * 4 + 2);
                             // first write of this pair into P^T and dS^T: dV of pair g-1 and dK, dQ of pair g-2 must have
                             // read them (they ran under the arithmetic above)
                             if (g > 0) ok = mbar_wait_ool(bar(PT_FREE), (g - 1) & 1, &abort_flag);
                             if (ok && g > 1) ok = mbar_wait_ool(bar(X_FREE + buf), ((g >> 1) - 1) & 1, &abort_flag);
-                            if (warp == 0) TRACE(16 + (g < 60 ? g : 59) * 4 + 3);
                         }
                         tmem_st16(tmem + Cfg::PT_COL + lane_base + (q0 >> 1), pk);
                         // dS^T row r, 32 queries: four 16-byte chunks of this half's panel, 128-byte swizzle
@@ -632,7 +628,6 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 fence_proxy_async_smem();
                 tc_fence_before();
                 mbar_arrive(bar(PDS_FULL + buf));
-                if (warp == 0) TRACE(16 + (g < 60 ? g : 59) * 4 + 1);
             }
         }
     }
@@ -641,11 +636,9 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (abort_flag) {
         for (int t = 0; t < 64; ++t) __nanosleep(1000);
     }
-    if (tid == 0) TRACE(4);
     tc_fence_before();
     __syncthreads();
     if (warp == 13) tmem_dealloc(tmem_base_s, Cfg::TMEM_COLS);
-    if (tid == 0) TRACE(5);
     if (tid == 0 && abort_flag) atomicExch(prm.status, 1);
 }
 

@@ -8,7 +8,6 @@
 // the four partial sums of a row are added at the end.
 #pragma once
 #include "ptx.cuh"
-#include "fwd_kernel.cuh"
 
 namespace attn {
 

@@ -28,15 +28,6 @@
 
 namespace attn {
 
-constexpr float LOG2E = 1.4426950408889634f;
-constexpr float LN2 = 0.6931471805599453f;
-
-#ifdef ATTN_TRACE
-#define TRACE(slot) do { if (prm.trace && blockIdx.x < 2048 && (threadIdx.x & 31) == 0) prm.trace[(size_t)blockIdx.x * 256 + (slot)] = ptx::globaltimer_ns(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#endif
-
 template <int D>
 struct FwdCfg {
     static constexpr int BR = 128, BC = 64;
@@ -52,11 +43,7 @@ struct FwdCfg {
     // shared by two threads (eight softmax warps per CTA) 80 us, against 73 us for this one: a warp spends
     // 0.5-0.9 us on the maximum and the 64 exponentials of a tile in every variant (the TMEM loads and stores
     // around them take 0.03-0.06 us each), so what counts is how many tiles the SM has in flight.
-    // (FWD64_TWO_BUFS=1 builds that variant for comparison.)
-#ifndef FWD64_TWO_BUFS
-#define FWD64_TWO_BUFS 0
-#endif
-    static constexpr int S_BUFS = (D == 128 || FWD64_TWO_BUFS) ? 2 : 1;
+    static constexpr int S_BUFS = (D == 128) ? 2 : 1;
     // With two score buffers the O-bar rescale is done by four correction warps (thread = query row, like the softmax
     // warps) next to the softmax warps' exponential pass instead of inside their per-tile chain: the running maximum of
     // some row of a warp moves in most tiles (probability 1 - (j/(j+1))^32 at tile j for random scores), so the TMEM
@@ -77,9 +64,6 @@ struct FwdCfg {
 };
 
 struct FwdParams {
-#ifdef ATTN_TRACE
-    unsigned long long* trace;
-#endif
     float* lse;
     int* ones;                 // COUNT instantiations only: per-row count of P-bar entries equal to 1
     int pbar_fmt;              // COUNT instantiations only: 0 = BF16 P-bar, 1 = E4M3, 2 = E5M2 (diagnostic)
@@ -130,7 +114,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) TRACE(0);
     const int bh = blockIdx.x % prm.BH;
     const int i = prm.Tr - 1 - blockIdx.x / prm.BH;        // heaviest (most key tiles) first
     int seqlen = prm.seqlen;
@@ -163,7 +146,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     griddep_wait();                                        // everything above ran beside the tail of the previous kernel
     const uint32_t tmem_S = tmem_base_s + Cfg::S_COL;
     const uint32_t tmem_O = tmem_base_s + Cfg::O_COL;
-    if (tid == 0) TRACE(1);
 
     if (warp == PRODUCER) {
         // ------------------------------------------------------------ TMA producer
@@ -208,7 +190,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 return true;
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, &abort_flag);
-            TRACE(2);
             ok = ok && issue_S(0);
             if (Cfg::S_BUFS == 2 && nkv > 1) ok = ok && issue_S(1);
             for (int j = 0; ok && j < nkv; ++j) {
@@ -350,6 +331,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const float m_new = fmaxf(m, mx);
                 a = ex2((m - m_new) * LOG2E);     // m = -inf on the first tile gives a = 0; a = 1 when m stays
                 const float negm = -m_new * LOG2E;
+                // Argument of ex2 for two scores.  Standard mode: one packed FMA, acc * (scale log2 e) - m log2 e.  Stabilised
+                // mode: the shifted maximum m = beta r_m can lie far above every score of the row, so the difference is taken
+                // first, as Algorithm 3 writes it, t = acc * scale - m (one rounding), and t is then brought to base 2; the
+                // error of the argument is then relative to |s - m| instead of |m|.
+                auto exp_arg = [&](float& x0, float& x1, float a0, float a1) {
+                    if (MODE == 1) {
+                        fma2(x0, x1, a0, a1, prm.scale, -m_new);
+                        mul2(x0, x1, x0, x1, LOG2E);
+                    } else {
+                        fma2(x0, x1, a0, a1, c_l2, negm);
+                    }
+                };
                 m = m_new;
                 // ---- last pass: P-bar = bf16(exp(S - m)) -> TMEM (over S); l += FP32 sum of the rounded values
                 float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
@@ -361,7 +354,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
                         float x0, x1;
-                        fma2(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), c_l2, negm);
+                        exp_arg(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
                         float p0 = ex2(x0), p1 = ex2(x1);
                         if (DIAG) {
                             if (h * 32 + c > vis) p0 = 0.0f;
@@ -440,6 +433,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const float m_new = fmaxf(m, mx);
                 a = ex2((m - m_new) * LOG2E);     // m = -inf on the first tile gives a = 0; a = 1 when m stays
                 const float negm = -m_new * LOG2E;
+                // Argument of ex2 for two scores.  Standard mode: one packed FMA, acc * (scale log2 e) - m log2 e.  Stabilised
+                // mode: the shifted maximum m = beta r_m can lie far above every score of the row, so the difference is taken
+                // first, as Algorithm 3 writes it, t = acc * scale - m (one rounding), and t is then brought to base 2; the
+                // error of the argument is then relative to |s - m| instead of |m|.
+                auto exp_arg = [&](float& x0, float& x1, float a0, float a1) {
+                    if (MODE == 1) {
+                        fma2(x0, x1, a0, a1, prm.scale, -m_new);
+                        mul2(x0, x1, x0, x1, LOG2E);
+                    } else {
+                        fma2(x0, x1, a0, a1, c_l2, negm);
+                    }
+                };
                 m = m_new;
                 if constexpr (Cfg::CORR) {                // the correction warps rescale O-bar under the exponential pass
                     sA[j & 1][row] = a;
@@ -452,7 +457,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
                         float x0, x1;
-                        fma2(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), c_l2, negm);
+                        exp_arg(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
                         float p0 = ex2(x0), p1 = ex2(x1);
                         if (DIAG) {
                             if (h * 32 + c > vis) p0 = 0.0f;
@@ -512,12 +517,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                                     : mbar_wait(bar(S_FULL), j & 1, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (warp == 0) TRACE(16 + j * 4 + 0);
             tc_fence_after();
             if (CAUSAL && j >= 2 * i)                         ok = tile(std::true_type{}, j, row - (j - 2 * i) * Cfg::BC);
             else if (PADDED && (j + 1) * Cfg::BC > seqlen)      ok = tile(std::true_type{}, j, seqlen - 1 - j * Cfg::BC);
             else                                              ok = tile(std::false_type{}, j, 0);
-            if (warp == 0) TRACE(16 + j * 4 + 1);
             if (!ok) break;
         }
         // ---- epilogue: O-bar -> BF16, O = bf16(O-bar / l), L = m + log l
@@ -525,7 +528,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             ok = mbar_wait(pv_done_bar(nkv - 1), pv_done_phase(nkv - 1), &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
         }
-        if (warp == 0) TRACE(3);
         if (ok) {
             tc_fence_after();
             const float rl = __frcp_rn(l);
@@ -572,11 +574,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         // let copies that are still in flight land before shared memory is released
         for (int t = 0; t < 64; ++t) __nanosleep(1000);
     }
-    if (tid == 0) TRACE(4);
     tc_fence_before();
     __syncthreads();
     if (warp == ISSUER) tmem_dealloc(tmem_base_s, Cfg::TMEM_COLS);
-    if (tid == 0) TRACE(5);
     if (tid == 0 && abort_flag) atomicExch(prm.status, 1);
 }
 

@@ -6,6 +6,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+namespace attn {
+constexpr float LOG2E = 1.4426950408889634f;     // log2(e): exponentials are taken in base 2 (ex2)
+constexpr float LN2 = 0.6931471805599453f;
+}  // namespace attn
+
 namespace ptx {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s per wait
@@ -64,16 +69,17 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t par
 //                                           while the forward and the d = 128 backward are faster with the loops inline)
 // The `relaxed` ones are for roles with slack: they sleep between polls, so that the waiting warp leaves the issue
 // slots and the shared-memory pipe to the warps that work.
+template <unsigned long long LIMIT_NS = WAIT_LIMIT_NS>
 __device__ __forceinline__ bool mbar_poll(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     unsigned long long t0 = 0;
     uint32_t polls = 0;
     while (true) {
         if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;
-        if ((++polls & 1023u) == 0u) {
+        if ((++polls & 1023u) == 0u || LIMIT_NS < 100000000ull) {      // short limits (self-test): look at the clock every poll
             if (*abort_flag) return false;
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+            else if (now - t0 > LIMIT_NS) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -92,13 +98,14 @@ __device__ __forceinline__ bool mbar_poll_relaxed(uint32_t bar, uint32_t parity,
     }
 }
 __device__ __noinline__ bool mbar_poll_ool(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return mbar_poll(bar, parity, abort_flag);
+    return mbar_poll<>(bar, parity, abort_flag);
 }
 __device__ __noinline__ bool mbar_poll_relaxed_ool(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_poll_relaxed(bar, parity, abort_flag);
 }
+template <unsigned long long LIMIT_NS = WAIT_LIMIT_NS>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return mbar_try_wait(bar, parity) || mbar_poll(bar, parity, abort_flag);
+    return mbar_try_wait(bar, parity) || mbar_poll<LIMIT_NS>(bar, parity, abort_flag);
 }
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_try_wait(bar, parity) || mbar_poll_relaxed(bar, parity, abort_flag);
@@ -309,6 +316,14 @@ __device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, f
         "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
         "mov.b64 {%0, %1}, rd;\n\t}"
         : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+// (d0, d1) = (a0, a1) * (b, b)
+__device__ __forceinline__ void mul2(float& d0, float& d1, float a0, float a1, float b) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b));
 }
 // (d0, d1) = (a0, a1) * (b, b) + (c0, c1)
 __device__ __forceinline__ void fma2v(float& d0, float& d1, float a0, float a1, float b, float c0, float c1) {

@@ -6,13 +6,18 @@ Tolerances (floating point):
   O against the BF16-emulating oracle:  within one BF16 ulp taken at the condition scale
                                         sum_t P|V| of the dot product (two correct FP32
                                         summation orders cannot agree more closely on outputs
-                                        that are small through cancellation).  At most 1e-4 of
-                                        the elements may be off by up to two ulp: O is rounded
-                                        twice (O-bar, then O-bar / l), and when ex2.approx puts a
-                                        P-bar value on the other side of a BF16 rounding boundary
-                                        than the oracle's exact exp (in the stabilised mode all
-                                        tied entries of a row share that value) each of the two
-                                        roundings can move by one ulp
+                                        that are small through cancellation).  Observed on the
+                                        GPU: no element beyond one ulp on C1, C2, C3 (standard
+                                        mode), C4 and every multi-tile shape; 6 of 2.1 M elements
+                                        on C5 (10 of 0.5 M on its head (0,0)) and 65 of 6.3 M on C3
+                                        in the stabilised mode reach two ulp (O is rounded twice,
+                                        O-bar and then O-bar / l, and each rounding can move by one
+                                        ulp when the FP32 sums differ in their last bits).  The bar:
+                                        at most 4e-5 of the elements beyond one ulp (twice the
+                                        largest fraction observed), none beyond two.
+                                        The strict count (one ulp at |O| itself, no condition
+                                        scale) is reported and bounded per configuration by about
+                                        twice its observed fraction (STRICT_BOUND below)
   L against the emulating oracle:       1e-4 + 1e-5 |L| on at least 98 % of the rows (same
                                         algorithm, FP32 noise only); a row where one P-bar entry
                                         rounds to the neighbouring BF16 value moves l by up to
@@ -36,6 +41,11 @@ pytestmark = pytest.mark.gpu
 
 MAX_ABS, REL_FRO = 2e-2, 1e-2
 L_TOL_FP64 = 2 ** -8 + 1e-4
+# Fraction of O elements that differ from the emulating oracle by more than one BF16 ulp of their own magnitude
+# (outputs that are small through cancellation).  Observed: C1 0, multi-tile shapes <= 3.9e-4, C2 3.9e-4, C3 1.6e-7
+# (standard) / 3.6e-5 (stabilised), C4 2.2e-3, C5 6e-4 to 2.0e-3 per head.  A regression that doubles these fails.
+STRICT_BOUND = {"C1": 2e-4, "C2": 8e-4, "C3": 8e-5, "C4": 4.5e-3, "C5": 4e-3, "shape": 1.1e-3}
+OBSERVED = []          # (label, violations, strict count, worst ratio, elements): printed at the end of the module
 
 
 def _gpu():
@@ -62,12 +72,23 @@ def _oracle_all(t, meta, mode):
     return dict(O=O, L=L, dQ=dQ, dK=dK, dV=dV, Oe=Oe, Le=Le, dQe=dqe, dKe=dke, dVe=dve, A=A)
 
 
-def _check_against_oracle(g, r, t, label):
+def _check_against_oracle(g, r, t, label, strict_key=None):
+    """Returns (violations of the one-ulp rule, strict count, worst ratio) of O against the emulating oracle."""
     # forward
     assert np.all(np.isfinite(as_f64(g["O"]))) and np.all(np.isfinite(g["L"])), label
-    assert max_abs(g["O"], r["O"]) <= MAX_ABS and rel_fro(g["O"], r["O"]) <= REL_FRO, label
+    if max_abs(r["Oe"], r["O"]) <= MAX_ABS and rel_fro(r["Oe"], r["O"]) <= REL_FRO:
+        assert max_abs(g["O"], r["O"]) <= MAX_ABS and rel_fro(g["O"], r["O"]) <= REL_FRO, label
+    else:
+        # the emulating oracle itself misses a bar on these inputs (|O| large enough that BF16 quantisation alone
+        # exceeds 2e-2 on some element): no implementation of these rounding points can meet it; bound the GPU by the
+        # oracle's own error instead
+        assert max_abs(g["O"], r["O"]) <= 1.25 * max_abs(r["Oe"], r["O"]), (label, max_abs(g["O"], r["O"]), max_abs(r["Oe"], r["O"]))
+        assert rel_fro(g["O"], r["O"]) <= 1.25 * rel_fro(r["Oe"], r["O"]), label
     viol, strict, worst = ulp_violations(g["O"], r["Oe"], r["A"])
-    assert viol <= 1e-4 * g["O"].size and worst <= 2.0, (label, viol, strict, worst)
+    OBSERVED.append((label, viol, strict, worst, g["O"].size))
+    assert viol <= 4e-5 * g["O"].size and worst <= 2.0, (label, viol, strict, worst)
+    if strict_key is not None:
+        assert strict <= max(1.0, STRICT_BOUND[strict_key] * g["O"].size), (label, viol, strict, worst)
     dL = np.abs(g["L"] - r["Le"])
     assert np.mean(dL > 1e-4 + 1e-5 * np.abs(r["Le"])) <= 0.02 and np.max(dL) <= L_TOL_FP64, label
     assert np.max(np.abs(g["L"] - r["L"])) <= L_TOL_FP64, label
@@ -99,13 +120,21 @@ def _check_against_oracle(g, r, t, label):
             # tied-maximum case, whose exact value is ~1e-5): bound the GPU by the oracle's own error
             assert max_abs(got, ref) <= 1.25 * max_abs(emu, ref), (label, n)
             assert rel_fro(got, ref) <= 1.25 * rel_fro(emu, ref), (label, n)
+    return viol, strict, worst
+
+
+def teardown_module(module):
+    # what was observed, for the record (shown with pytest -s or -rA)
+    for label, viol, strict, worst, size in OBSERVED:
+        print(f"[O vs emulating oracle] {label}: beyond one ulp {viol}, strict {strict} of {size} ({strict / size:.2e}), worst {worst:.2f}")
 
 
 @pytest.mark.parametrize("mode", [0, 1])
 def test_c1_single_tile(mode):
     t, m = ai.make("C1")
     g = _gpu().run_fwd_bwd(t, m, mode)
-    _check_against_oracle(g, _oracle_all(t, m, mode), t, f"C1 mode {mode}")
+    viol, strict, worst = _check_against_oracle(g, _oracle_all(t, m, mode), t, f"C1 mode {mode}", "C1")
+    assert viol == 0
 
 
 @pytest.mark.parametrize("B,H,N,d,causal,mode", [
@@ -124,7 +153,9 @@ def test_multi_tile_shapes(B, H, N, d, causal, mode):
     t = ai.gaussian(B, H, N, d, seed=100 + N + d + B)
     m = dict(B=B, H=H, N=N, d=d, causal=causal, alpha=d ** -0.5)
     g = _gpu().run_fwd_bwd(t, m, mode)
-    _check_against_oracle(g, _oracle_all(t, m, mode), t, f"{B}x{H}x{N}x{d} causal={causal} mode={mode}")
+    viol, strict, worst = _check_against_oracle(g, _oracle_all(t, m, mode), t,
+                                                f"{B}x{H}x{N}x{d} causal={causal} mode={mode}", "shape")
+    assert viol == 0
 
 
 def test_results_are_reproducible_run_to_run():
@@ -184,8 +215,8 @@ def test_mitigation_parameters_are_honoured():
 
 @pytest.fixture(scope="module")
 def c3_runs():
-    # tied-maximum stress case, all 12 heads of one batch entry (the recipe is per head)
-    t, m = ai.make("C3", B=2)
+    # tied-maximum stress case at the configuration's size: B = 8, all 96 heads (the recipe is per head)
+    t, m = ai.make("C3")
     O, L = oracle.ref_fwd(t["q"], t["k"], t["v"], True, m["alpha"])
     out = {}
     for mode in (0, 1):
@@ -207,15 +238,17 @@ def test_c3_rounding_bias_statistic(c3_runs):
     assert e0["E_O"] > 2e-4 and e0["E_delta"] > 5e-4
     assert abs(g0["E_O"] - e0["E_O"]) <= 5e-4 * abs(e0["E_O"])
     assert abs(g0["E_delta"] - e0["E_delta"]) <= 5e-4 * abs(e0["E_delta"])
-    # stabilised mode: an order of magnitude smaller.  Here every tied entry of a row shares one
-    # P-bar value p = bf16(exp(-(beta-1) r_m)) with |(beta-1) r_m| up to 40: an FP32 ex2 of an
-    # argument of magnitude ~58 is only good to ~20 ulp, so now and then p lands on the other side of
-    # a BF16 rounding boundary than the oracle's exactly rounded exp, which moves every output of the
-    # rows with that (head, r_m) by up to an ulp: about 3e-6 on this mean per such event.  The
-    # statistic is therefore compared on the scale of the standard-mode bias, to 0.5 % of it.
+    # stabilised mode: an order of magnitude smaller, and compared on the scale of the standard-mode bias.
+    # Observed at B = 8 (96 heads, 63,106 tied rows): E_O 4.549e-5 on the GPU against 4.655e-5 (oracle), E_delta 1.499e-4
+    # against 1.539e-4: 1.7e-3 and 2.0e-3 of the standard-mode values.  No P-bar entry differs from the oracle's (L agrees
+    # to 7.6e-6 on all 98,304 rows; one flipped entry of a tied row would move it by 4e-3); what differs is the FP32
+    # accumulation of O-bar: here a tied row sums k = 2 or 4 equal products p v with p = bf16(exp(-(beta-1) r_m)), 16-bit
+    # products whose FP32 sum the tensor core does not round as a sequence of IEEE additions, and 2,112 of the 98,304
+    # rows hold an element whose O-bar then rounds to the other BF16 neighbour (362 rows in the standard mode, where
+    # p = 1 and the sums are exact).  The bar is 3e-3 of the standard-mode statistic.
     assert abs(g1["E_O"]) <= 0.1 * abs(g0["E_O"]) and abs(g1["E_delta"]) <= 0.1 * abs(g0["E_delta"])
-    assert abs(g1["E_O"] - e1["E_O"]) <= 5e-3 * abs(e0["E_O"])
-    assert abs(g1["E_delta"] - e1["E_delta"]) <= 5e-3 * abs(e0["E_delta"])
+    assert abs(g1["E_O"] - e1["E_O"]) <= 3e-3 * abs(e0["E_O"])
+    assert abs(g1["E_delta"] - e1["E_delta"]) <= 3e-3 * abs(e0["E_delta"])
 
 
 def test_c3_outputs_and_gradients(c3_runs):
@@ -228,7 +261,9 @@ def test_c3_outputs_and_gradients(c3_runs):
         de = oracle.emu_delta(Oe, t["dO"])
         dqe, dke, dve = oracle.emu_bwd(t["q"], t["k"], t["v"], t["dO"], Le, de, True, m["alpha"])
         r = dict(O=O, L=L, dQ=dQ, dK=dK, dV=dV, Oe=Oe, Le=Le, dQe=dqe, dKe=dke, dVe=dve, A=A)
-        _check_against_oracle(g, r, t, f"C3 mode {mode}")
+        viol, strict, worst = _check_against_oracle(g, r, t, f"C3 mode {mode}", "C3")
+        if mode == 0:
+            assert viol == 0
 
 
 def _sampled_heads_check(name, heads, mode, B=None):
@@ -243,7 +278,10 @@ def _sampled_heads_check(name, heads, mode, B=None):
         sub = {n: np.ascontiguousarray(t[n][b:b + 1, h:h + 1]) for n in ("q", "k", "v", "dO")}
         ms = dict(m, B=1, H=1)
         gs = {n: np.ascontiguousarray(g[n][b:b + 1, h:h + 1]) for n in g}
-        _check_against_oracle(gs, _oracle_all(sub, ms, mode), sub, f"{name} head ({b},{h}) mode {mode}")
+        viol, strict, worst = _check_against_oracle(gs, _oracle_all(sub, ms, mode), sub,
+                                                    f"{name} head ({b},{h}) mode {mode}", name)
+        if name != "C5":
+            assert viol == 0
 
 
 @pytest.mark.parametrize("mode", [0, 1])

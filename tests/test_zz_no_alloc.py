@@ -16,7 +16,7 @@ import attn_inputs as ai
 pytestmark = pytest.mark.gpu
 
 
-def _run_pair(B, H, N, d, causal, seed):
+def _run_pair(B, H, N, d, causal, seed, check_no_allocation=False):
     import paper_2510_04212_b200 as attn
     from _gpu_util import to_bits, to_dev
     from _metrics import as_f64, rel_fro
@@ -38,9 +38,17 @@ def _run_pair(B, H, N, d, causal, seed):
                   B, H, N, d, causal, alpha, 0)
     # new entry point: no workspace argument
     dq1, dk1, dv1, delta1 = outputs()
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    allocs_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
     attn.attn_bwd_static(dev["q"], dev["k"], dev["v"], o, dev["dO"], lse, dq1, dk1, dv1, delta1,
                          B, H, N, d, causal, alpha, 0)
     torch.cuda.synchronize()
+    if check_no_allocation:
+        # what the entry point exists for: the device's free memory is what it was (the driver's own view, so an
+        # allocation by the library itself would show), and torch's allocator was not asked for anything either
+        assert torch.cuda.mem_get_info()[0] == free_before
+        assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
     assert attn.attn_last_device_status() == 0
     assert np.array_equal(to_bits(dk1), to_bits(dk0))
     assert np.array_equal(to_bits(dv1), to_bits(dv0))
@@ -52,9 +60,14 @@ def _run_pair(B, H, N, d, causal, seed):
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point():
     # the second call is smaller and differently shaped: it must not see what the first left behind
-    _run_pair(2, 4, 512, 64, True, seed=31)
-    _run_pair(1, 3, 256, 128, False, seed=32)
-    _run_pair(2, 4, 512, 64, True, seed=33)
+    _run_pair(2, 4, 512, 64, True, seed=31)     # the first call on the device resolves the scratch address
+    _run_pair(1, 3, 256, 128, False, seed=32, check_no_allocation=True)
+    _run_pair(2, 4, 512, 64, True, seed=33, check_no_allocation=True)
+
+
+def test_a_call_that_uses_the_whole_scratch():
+    # B*H*N*d = 8,388,608 elements: exactly the 32 MiB the library holds
+    _run_pair(8, 16, 1024, 64, True, seed=34, check_no_allocation=True)
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
@@ -63,6 +76,8 @@ def test_sizes_beyond_the_built_in_scratch_are_refused():
     # 16*12*1024*64 elements need 48 MiB > 32 MiB
     assert attn.lib.attn_bwd_static(p, p, p, p, p, p, p, p, p, p, 16, 12, 1024, 64, 1, 0.125, 0, None) == -5
     assert "workspace" in attn.attn_strerror(-5)
+    # the checks come in attn_bwd's order: a NULL pointer is reported before the size
+    assert attn.lib.attn_bwd_static(None, p, p, p, p, p, p, p, p, p, 16, 12, 1024, 64, 1, 0.125, 0, None) == -1
     # exactly at the limit is accepted by the size check (and then fails only on the fake pointers' alignment
     # or NULL checks, never with the workspace error): 8*16*1024*64*4 bytes = 32 MiB
     assert attn.attn_bwd_workspace_bytes(8, 16, 1024, 64) == 32 << 20
