@@ -5,20 +5,35 @@
 // running across item boundaries, so the loads, the first MMAs and the output stores of neighbouring
 // items overlap instead of adding a prologue and a tail per item.
 //
-// Per (i, j) pair, five tcgen05 MMAs (FP32 accumulators in TMEM):
-//   group A   S^T  = K_j Q_i^T     dP^T = V_j dO_i^T
-//   group B   dV  += P^T dO_i      dK  += dS^T Q_i      dQ_i = dS K_j
+// Per (i, j) pair, five products on the tensor cores (FP32 accumulators in TMEM), 32 tcgen05.mma in all:
+//   group A   S^T  = K_j Q_i^T     dP^T = V_j dO_i^T                         (8 instructions, N = 128)
+//   group B   dQ_i = dS K_j        dV  += P^T dO_i      dK  += dS^T Q_i      (24 instructions, N = 64)
 // TMEM (512 columns): S^T [0,128) | dP^T [128,256) | P^T (BF16) [256,320) | dV [320,384) |
-// dK [384,448) | dQ [448,512).  The compute warps release S^T / dP^T as soon as they have loaded them
-// into registers (half way through their work on the pair), so A of the next pair runs under the second
-// half; P^T has its own columns and dS^T is double-buffered in shared memory.
+// dK [384,448) | dQ [448,512).
+//
+// What bounds this kernel is the rate at which an SM's tensor front end takes tcgen05 instructions: one
+// tcgen05.mma OR tcgen05.commit per 50-60 clocks, whichever thread issues it (measured: a stream of N = 64
+// MMAs retires one per 46-49 clocks, N = 128 one per 63; eight N = 64 MMAs issued into an idle pipe take 514
+// clocks, and every commit after them another 45-54).  So the kernel is built to issue as few of them as
+// possible: 32 MMAs and 3 commits per pair (S^T/dP^T ready; dV and dQ
+// done; dK done), plus two commits per work item (V free, K free).  A pair then costs about 1.8 k
+// clocks of front-end time, which the element-wise work of the compute warps (also about 1.8 k clocks per
+// pair) runs beside.
 //
 // Warps: 0-7 compute (thread = key row x 64 query columns: warps 0-3 take query columns [0,64), warps 4-7
 // [64,128)); 8-11 drain (dQ tiles and, once per item, dV / dK: TMEM -> shared-memory staging; also the
-// final dQ conversion described below); 12 TMA producer; 13 and 14 MMA issuers (13: group A and dV,
-// 14: dK and dQ; one thread issues about one MMA per 100 clocks, the tensor pipe retires one in 50-70);
-// 15 staging consumer (TMA reduce-add of dQ tiles into the FP32 accumulator in global memory, TMA stores
-// of dV / dK, arrival counting).
+// final dQ conversion described below); 12 TMA producer; 13 MMA issuer for group A; 14 MMA issuer for group B;
+// 15 staging consumer
+// (TMA reduce-add of dQ tiles into the FP32 accumulator in global memory, TMA stores of dV / dK, arrival
+// counting).  Barriers that whole warps arrive on count one arrival per warp (lane 0, after __syncwarp).
+//
+// Order of the issuer's stream inside a work item: A(g+1) as soon as the compute warps hold S^T, dP^T of
+// pair g in registers (half way through their work on it), then, when they have finished pair g, dV(g)
+// and dQ(g) under one commit (the compute warps' next P^T, the drain and, on the last pair of an item,
+// the reload of K wait for it), then dK(g).
+// The staging buffer is two 16 KB panels with a full / free barrier each, so that the drain writes one
+// panel while the TMA engine still reads the other (an SM's FP32 reduce-adds leave at 30-50 GB/s: the
+// 32 KB of a pair take about as long as the pair itself).
 //
 // dQ leaves the kernel finished: the first 32-bit word of every 128-row dQ output tile serves as an
 // arrival counter (cleared by the preprocess kernel) until the tile is written.  After its reduce-adds
@@ -151,25 +166,33 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t sQ0 = sV + Cfg::TILE_BYTES;                    // QS stages
     const uint32_t sdO0 = sQ0 + Cfg::QS * Cfg::TILE_BYTES;        // QS stages
     const uint32_t sX0 = sdO0 + Cfg::QS * Cfg::TILE_BYTES;        // two buffers
-    const uint32_t sStg = sX0 + 2 * Cfg::X_BYTES;
+    const uint32_t sStg = sX0 + 2 * Cfg::X_BYTES;                 // two panels of TILE_BYTES
     uint8_t* sX_ptr = sm + (2 + 2 * Cfg::QS) * Cfg::TILE_BYTES;
     uint8_t* sStg_ptr = sX_ptr + 2 * Cfg::X_BYTES;
 
     // Barriers.  g = running pair count of this CTA (over all its items), w = running item count, n = running
     // staging step count (one per pair plus one per item).  Unless noted, a barrier completes one phase per g.
-    //   K_FULL, V_FULL (per w)      TMA landed                          K_FREE (per w, 2 commits), V_FREE (per w): MMAs done reading
-    //   QDO_FULL / QDO_EMPTY [QS]   Q_i, dO_i ring (EMPTY: both issuers' commits)
-    //   SDP_FULL                    A(g) done                           SDP_FREE: compute warps hold S^T, dP^T of g in registers
-    //   PDS_FULL [2]                P^T in TMEM, dS^T in X[g & 1]       PT_FREE: dV(g) done; X_FREE [2]: dK(g), dQ(g) done
-    //   DQ_FULL / DQ_EMPTY          dQ tile in TMEM / read by the drain
-    //   DKV_DONE (per w, 2 commits) dV, dK of the item complete         DKV_FREE (per w): read by the drain
-    //   STG_FULL / STG_FREE (per n) staging written / read by TMA       VEC_FULL [2]: per-query vectors of g landed (bulk copies)
+    // A wait on a barrier costs a shared-memory round trip of some 200 clocks while MMAs run (their operand fetch has
+    // the shared-memory pipe), so each MMA issuer waits on ONE barrier per pair, which collects every arrival it needs:
+    //   A_READY [QS] (per stage)    Q_i, dO_i of pair g landed (TMA) AND the compute warps hold S^T, dP^T of pair g - 1 in
+    //                               registers (8 warp arrivals; before the first pair they arrive once unconditionally)
+    //   B_READY                     P^T in TMEM and dS^T in X[g & 1] (8 compute-warp arrivals) AND the drain has read dQ of
+    //                               pair g - 1 (4 drain-warp arrivals; once unconditionally before the first pair)
+    //   K_FULL, V_FULL (per w)      TMA landed                          K_FREE, V_FREE (per w): last dQ / last A of the item done
+    //   SDP_FULL                    A(g) done                           VEC_FULL [2]: per-query vectors of g landed (bulk copies)
+    //   PDS_FULL [2]                the compute warps have finished pair g (index g & 1, phase (g >> 1) & 1): only the
+    //                               producer waits here, for pair g - 2, before it reuses that pair's vector buffer
+    //   DQ_FULL                     dV(g) and dQ(g) done: the dQ tile is in TMEM and P^T may be overwritten (with everything
+    //                               issued before them: the dS^T buffer of pair g - 1 is free too)
+    //   B_DONE [2]                  dK(g) and everything issued before it complete: the Q / dO stage of g is free; on the
+    //                               last pair of an item dV, dK are final (index g & 1, phase (g >> 1) & 1: the producer
+    //                               looks three pairs back and may be late by a pair after waiting for K)
+    //   DKV_FREE (per w)            dV, dK read by the drain
+    //   STG_FULL / STG_FREE [2]     (per n, one pair per staging panel) panel written / read by TMA
     //   FIN                         last arrival verdicts written
-    // PDS_FULL and X_FREE exist once per dS^T buffer (index = g & 1): issuer 14 may run up to two pairs behind the
-    // compute warps (it also waits for the drain), which a single barrier's phase parity could not tell apart.
-    enum { K_FULL = 0, V_FULL = 1, K_FREE = 2, V_FREE = 3, QDO_FULL = 4, QDO_EMPTY = 7, SDP_FULL = 10, SDP_FREE = 11,
-           PDS_FULL = 12, PT_FREE = 14, X_FREE = 15, DQ_FULL = 17, DQ_EMPTY = 18, DKV_DONE = 19, DKV_FREE = 20,
-           STG_FULL = 21, STG_FREE = 22, VEC_FULL = 23, FIN = 25, NBARS = 26 };
+    enum { K_FULL = 0, V_FULL = 1, K_FREE = 2, V_FREE = 3, A_READY = 4, SDP_FULL = 7, B_READY = 8,
+           PDS_FULL = 9, B_DONE = 11, DQ_FULL = 13, DKV_FREE = 14,
+           STG_FULL = 15, STG_FREE = 17, VEC_FULL = 19, FIN = 21, NBARS = 22 };
     uint8_t* misc = sm + Cfg::TILES_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                           // NBARS x 8 bytes (256 reserved)
     float (*sNegL)[128] = reinterpret_cast<float (*)[128]>(misc + 256);           // [2][128]: -L * log2(e) per query of the tile
@@ -187,9 +210,10 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     if (tid == 0) {
         for (int b = 0; b < NBARS; ++b) {
             uint32_t cnt = 1;
-            if (b == SDP_FREE || b == PDS_FULL || b == PDS_FULL + 1) cnt = 256;
-            if (b == DQ_EMPTY || b == STG_FULL || b == DKV_FREE) cnt = 128;
-            if ((b >= QDO_EMPTY && b < QDO_EMPTY + Cfg::QS) || b == DKV_DONE || b == K_FREE) cnt = 2;   // both MMA issuers
+            if (b == PDS_FULL || b == PDS_FULL + 1) cnt = 8;                                    // one arrival per compute warp
+            if (b >= A_READY && b < A_READY + Cfg::QS) cnt = 9;                                 // ... plus the producer's (with the TMA bytes)
+            if (b == B_READY) cnt = 12;                                                         // compute warps and drain warps
+            if (b == DKV_FREE || b == STG_FULL || b == STG_FULL + 1) cnt = 4;                   // one per drain warp
             mbar_init(bar(b), cnt);
         }
         abort_flag = 0;
@@ -217,19 +241,20 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int kvrow0 = item.bh * prm.N + item.j * 128;
                 // V is free once the last A of the previous item has run, K only after its last dQ: V, the first
                 // Q / dO pair, then K
-                if (w > 0) ok = mbar_wait_relaxed_ool(bar(V_FREE), (w - 1) & 1, &abort_flag);
+                if (w > 0) ok = mbar_wait_ool(bar(V_FREE), (w - 1) & 1, &abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(bar(V_FULL), Cfg::TILE_BYTES);
                 tma_load_2d(sV, &tmV, bar(V_FULL), 0, kvrow0);
                 BwdPairPos<GENERAL> pos;
                 for (int it = 0; it < item.nq; ++it, ++g, pos.next(item)) {
-                    const int st = g % Cfg::QS, ph = (g / Cfg::QS) & 1;
-                    ok = mbar_wait_relaxed_ool(bar(QDO_EMPTY + st), ph ^ 1, &abort_flag);
+                    const int st = g % Cfg::QS;
+                    // the stage was last used by pair g - QS: free when that pair's dV, dK have run
+                    if (g >= Cfg::QS) ok = mbar_wait_relaxed_ool(bar(B_DONE + ((g - Cfg::QS) & 1)), ((g - Cfg::QS) >> 1) & 1, &abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(bar(QDO_FULL + st), 2 * Cfg::TILE_BYTES);
+                    mbar_expect_tx(bar(A_READY + st), 2 * Cfg::TILE_BYTES);
                     const int qrow = pos.row(item, prm);
-                    tma_load_2d(sQ0 + st * Cfg::TILE_BYTES, &tmQ, bar(QDO_FULL + st), 0, qrow);
-                    tma_load_2d(sdO0 + st * Cfg::TILE_BYTES, &tmdO, bar(QDO_FULL + st), 0, qrow);
+                    tma_load_2d(sQ0 + st * Cfg::TILE_BYTES, &tmQ, bar(A_READY + st), 0, qrow);
+                    tma_load_2d(sdO0 + st * Cfg::TILE_BYTES, &tmdO, bar(A_READY + st), 0, qrow);
                     {   // per-query vectors of this pair, into the buffer the compute warps used two pairs ago
                         const int vb = g & 1;
                         if (g >= 2) ok = mbar_wait_relaxed_ool(bar(PDS_FULL + vb), ((g - 2) >> 1) & 1, &abort_flag);
@@ -240,7 +265,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         bulk_load_1d(smem_u32(&sDelta[vb][0]), vec + VEC_NDELTA_OFFSET, 512, bar(VEC_FULL + vb));
                     }
                     if (it == 0) {
-                        if (w > 0) ok = mbar_wait_relaxed_ool(bar(K_FREE), (w - 1) & 1, &abort_flag);
+                        if (w > 0) ok = mbar_wait_ool(bar(K_FREE), (w - 1) & 1, &abort_flag);
                         if (!ok) break;
                         mbar_expect_tx(bar(K_FULL), Cfg::TILE_BYTES);
                         tma_load_2d(sK, &tmK, bar(K_FULL), 0, kvrow0);
@@ -250,85 +275,43 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         __syncwarp();
     } else if (warp == 13) {
-        // ------------------------------------------------------------ MMA issuer 1: group A and dV
+        // ------------------------------------------------------------ MMA issuer 1: group A (S^T, dP^T), one pair ahead
         if (lane == 0) {
-            constexpr uint32_t idesc_T = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: both operands K-major
-            constexpr uint32_t idesc_KN = make_idesc_bf16(128, D, 0, 1);    // dV: A from TMEM, B MN-major
+            constexpr uint32_t idesc_T = make_idesc_bf16(128, 128, 0, 0);   // both operands K-major
             // descriptors: only the start-address field (low word, 16-byte units) changes in the loops
             const uint64_t dK_k = make_smem_desc(sK, 16, 1024);             // K_j, K-major (rows of d)
             const uint64_t dV_k = make_smem_desc(sV, 16, 1024);
             const uint64_t dQ_k0 = make_smem_desc(sQ0, 16, 1024);
             const uint64_t ddO_k0 = make_smem_desc(sdO0, 16, 1024);
-            const uint64_t ddO_mn0 = make_smem_desc(sdO0, Cfg::TILE_BYTES, 1024);
-
-            // group A of pair gn; `last`: it is the last pair of its item (V and, for this issuer, K are free after it)
-            auto issue_A = [&](int gn, bool last) -> bool {
-                const int st = gn % Cfg::QS, ph = (gn / Cfg::QS) & 1;
-                if (!mbar_wait_ool(bar(QDO_FULL + st), ph, &abort_flag)) return false;
-                tc_fence_after();
-                const uint64_t so = static_cast<uint64_t>((st * Cfg::TILE_BYTES) >> 4);
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem + Cfg::DP_COL, dV_k + ((k * 32) >> 4), ddO_k0 + so + ((k * 32) >> 4), idesc_T, k > 0);
-                if (last) mma_commit(bar(V_FREE));
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem + Cfg::ST_COL, dK_k + ((k * 32) >> 4), dQ_k0 + so + ((k * 32) >> 4), idesc_T, k > 0);
-                mma_commit(bar(SDP_FULL));
-                if (last) mma_commit(bar(K_FREE));
-                return true;
-            };
-
-            // One code copy of group A and one of dV (instruction-cache footprint): the loop walks the pairs with a
-            // one-pair lookahead; step g issues A(g + 1) and dV(g).  Within an item A(g + 1) goes first (as soon as
-            // the compute warps hold S^T, dP^T of pair g in registers); across an item boundary dV(g) goes first,
-            // because the next item's K arrives only after this item's last dQ.
             bool ok = true;
-            BwdItem nxt;
-            int wn = 0, itn = 0;                          // position of pair g + 1
-            int en = 0;                                   // enumeration cursor of the lookahead
-            bool have_n = bwd_item<CAUSAL, GENERAL>(en, prm, nxt);
-            int wc = 0, itc = 0, nqc = 0;                 // position of pair g
-            for (int g = -1; ok; ++g) {
-                const int a_phase = (have_n && itn != 0) ? 0 : 1;
-#pragma unroll 1
-                for (int phase = 0; ok && phase < 2; ++phase) {
-                    if (phase == a_phase) {
-                        if (!have_n) continue;
-                        if (g >= 0) ok = mbar_wait_ool(bar(SDP_FREE), g & 1, &abort_flag);
-                        if (ok && itn == 0)
-                            ok = mbar_wait_ool(bar(V_FULL), wn & 1, &abort_flag) &&
-                                 mbar_wait_ool(bar(K_FULL), wn & 1, &abort_flag);
-                        ok = ok && issue_A(g + 1, itn == nxt.nq - 1);
-                    } else {
-                        if (g < 0) continue;
-                        ok = mbar_wait_ool(bar(PDS_FULL + (g & 1)), (g >> 1) & 1, &abort_flag);
-                        if (ok && itc == 0 && wc > 0) ok = mbar_wait_ool(bar(DKV_FREE), (wc - 1) & 1, &abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const int st = g % Cfg::QS;
-                        const uint64_t so = static_cast<uint64_t>((st * Cfg::TILE_BYTES) >> 4);
-                        // dV += P^T dO_i : A = P^T in TMEM, B = dO_i with d contiguous (MN-major), 16 queries per step
-                        mma_ts(tmem + Cfg::DV_COL, tmem + Cfg::PT_COL, ddO_mn0 + so, idesc_KN, (itc > 0) ? 1u : 0u);
+            int g = 0;
+            for (int w = 0, e = 0; ok && bwd_item<CAUSAL, GENERAL>(e, prm, item); ++w) {
+                const int nq = item.nq;
+                ok = mbar_wait_ool(bar(V_FULL), w & 1, &abort_flag) && mbar_wait_ool(bar(K_FULL), w & 1, &abort_flag);
+                for (int it = 0; ok && it < nq; ++it, ++g) {
+                    const int st = g % Cfg::QS, ph = (g / Cfg::QS) & 1;
+                    ok = mbar_wait_ool(bar(A_READY + st), ph, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t so = static_cast<uint64_t>((st * Cfg::TILE_BYTES) >> 4);
 #pragma unroll
-                        for (int k = 1; k < 8; ++k)
-                            mma_ts(tmem + Cfg::DV_COL, tmem + Cfg::PT_COL + k * 8, ddO_mn0 + so + ((k * 2048) >> 4), idesc_KN, 1u);
-                        mma_commit(bar(PT_FREE));
-                        mma_commit(bar(QDO_EMPTY + st));
-                        if (itc == nqc - 1) mma_commit(bar(DKV_DONE));
-                    }
+                    for (int k = 0; k < D / 16; ++k)
+                        mma_ss(tmem + Cfg::DP_COL, dV_k + ((k * 32) >> 4), ddO_k0 + so + ((k * 32) >> 4), idesc_T, k > 0);
+                    if (it == nq - 1) mma_commit(bar(V_FREE));                // last pair of the item: V may be reloaded
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k)
+                        mma_ss(tmem + Cfg::ST_COL, dK_k + ((k * 32) >> 4), dQ_k0 + so + ((k * 32) >> 4), idesc_T, k > 0);
+                    mma_commit(bar(SDP_FULL));
                 }
-                if (!have_n) break;
-                wc = wn; itc = itn; nqc = nxt.nq;
-                if (++itn == nxt.nq) { itn = 0; ++wn; have_n = bwd_item<CAUSAL, GENERAL>(en, prm, nxt); }
             }
         }
         __syncwarp();
     } else if (warp == 14) {
-        // ------------------------------------------------------------ MMA issuer 2: dK and dQ
+        // ------------------------------------------------------------ MMA issuer 2: group B (dV, dQ, dK)
         if (lane == 0) {
-            constexpr uint32_t idesc_KN = make_idesc_bf16(128, D, 0, 1);    // dK: A K-major, B MN-major
+            constexpr uint32_t idesc_KN = make_idesc_bf16(128, D, 0, 1);    // dV (A from TMEM), dK (A K-major): B MN-major
             constexpr uint32_t idesc_NN = make_idesc_bf16(128, D, 1, 1);    // dQ: A MN-major, B MN-major
+            const uint64_t ddO_mn0 = make_smem_desc(sdO0, Cfg::TILE_BYTES, 1024);
             const uint64_t dK_mn = make_smem_desc(sK, Cfg::TILE_BYTES, 1024);    // K_j as [key][d], MN-major B
             const uint64_t dQ_mn0 = make_smem_desc(sQ0, Cfg::TILE_BYTES, 1024);
             const uint64_t dX_k0 = make_smem_desc(sX0, 16, 1024);           // dS^T rows (queries contiguous): K-major A
@@ -337,50 +320,44 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             int g = 0;
             for (int w = 0, e = 0; ok && bwd_item<CAUSAL, GENERAL>(e, prm, item); ++w) {
                 const int nq = item.nq;
-                ok = mbar_wait_ool(bar(K_FULL), w & 1, &abort_flag);
+                // the accumulators of a new item overwrite dV, dK: the drain must have read the previous item's
+                if (w > 0) ok = mbar_wait_ool(bar(DKV_FREE), (w - 1) & 1, &abort_flag);
                 for (int it = 0; ok && it < nq; ++it, ++g) {
-                    const int st = g % Cfg::QS, ph = (g / Cfg::QS) & 1;
-                    ok = mbar_wait_ool(bar(PDS_FULL + (g & 1)), (g >> 1) & 1, &abort_flag) &&
-                         mbar_wait_ool(bar(QDO_FULL + st), ph, &abort_flag);
-                    if (ok && it == 0 && w > 0) ok = mbar_wait_ool(bar(DKV_FREE), (w - 1) & 1, &abort_flag);
+                    const int st = g % Cfg::QS;
+                    ok = mbar_wait_ool(bar(B_READY), g & 1, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t so = static_cast<uint64_t>((st * Cfg::TILE_BYTES) >> 4);
                     const uint64_t xo = static_cast<uint64_t>(((g & 1) * Cfg::X_BYTES) >> 4);
-                    // dK += dS^T Q_i : A = dS^T rows (K-major: 4 steps per 64-query panel), B = Q_i MN-major
-                    mma_ss(tmem + Cfg::DK_COL, dX_k0 + xo, dQ_mn0 + so, idesc_KN, (it > 0) ? 1u : 0u);
-#pragma unroll
-                    for (int k = 1; k < 8; ++k)
-                        mma_ss(tmem + Cfg::DK_COL, dX_k0 + xo + (((k >> 2) * Cfg::TILE_BYTES + (k & 3) * 32) >> 4),
-                               dQ_mn0 + so + ((k * 2048) >> 4), idesc_KN, 1u);
-                    if (g > 0) {
-                        ok = mbar_wait_ool(bar(DQ_EMPTY), (g - 1) & 1, &abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                    }
-                    // dQ_i = dS K_j : A = the same dS^T buffer read as (M = query, K = key), B = K_j MN-major
+                    // dQ_i = dS K_j : A = the dS^T buffer read as (M = query, K = key), B = K_j MN-major
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
                         mma_ss(tmem + Cfg::DQ_COL, dX_mn0 + xo + ((k * 2048) >> 4), dK_mn + ((k * 2048) >> 4), idesc_NN, k > 0);
-                    mma_commit(bar(DQ_FULL));
-                    mma_commit(bar(X_FREE + (g & 1)));                    // this dS^T buffer has been read
-                    mma_commit(bar(QDO_EMPTY + st));
-                    if (it == nq - 1) {
-                        mma_commit(bar(DKV_DONE));
-                        mma_commit(bar(K_FREE));
-                    }
+                    if (it == nq - 1) mma_commit(bar(K_FREE));                 // last pair of the item: K may be reloaded
+                    // dV += P^T dO_i : A = P^T in TMEM, B = dO_i with d contiguous (MN-major), 16 queries per step
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mma_ts(tmem + Cfg::DV_COL, tmem + Cfg::PT_COL + k * 8, ddO_mn0 + so + ((k * 2048) >> 4), idesc_KN,
+                               (it > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(bar(DQ_FULL));                                  // dQ(g) and dV(g): dQ tile ready, P^T free
+                    // dK += dS^T Q_i : A = dS^T rows (K-major: 4 steps per 64-query panel), B = Q_i MN-major
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss(tmem + Cfg::DK_COL, dX_k0 + xo + (((k >> 2) * Cfg::TILE_BYTES + (k & 3) * 32) >> 4),
+                               dQ_mn0 + so + ((k * 2048) >> 4), idesc_KN, (it > 0 || k > 0) ? 1u : 0u);
+                    mma_commit(bar(B_DONE + (g & 1)));
                 }
             }
         }
         __syncwarp();
     } else if (warp == 15) {
-        // ------------------------------------------------------------ staging consumer: TMA out of the staging buffer, arrival counts
+        // ------------------------------------------------------------ staging consumer: TMA out of the staging panels, arrival counts
         if (lane == 0) {
             // Arrival counting, two steps behind the TMA issue so that neither the completion of the reduce-adds nor
             // the atomic's round trip holds up the next staging step:
-            //   step n, after its STG_FREE arrival:  (1) the atomic issued in step n-1 (for step n-2) has returned by now:
-            //   turn it into the verdict on step n-2;  (2) the bulk group of step n-1 is the only older one: wait for it,
-            //   then issue the atomic for step n-1 without touching its result.
+            //   step n, after its two bulk groups are issued:  (1) the atomic issued in step n-1 (for step n-2) has returned by
+            //   now: turn it into the verdict on step n-2;  (2) the two groups of step n are the only ones that may still be
+            //   incomplete: wait for everything older (step n-1), then issue the atomic for step n-1 without touching its result.
             // The atomic releases this CTA's completed reduce-adds; the CTA that brings a tile's counter to the number
             // of key tiles that see the tile acquires the others' and finishes the tile.
             bool ok = true;
@@ -388,14 +365,15 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             int prev_t = -1, prev_i = 0, prev_Tr = 0;             // dQ tile of step n-1 (-1: it was a dV / dK step)
             int pend_t = -1;                                      // dQ tile of step n-2 whose atomic is in flight (-1: none)
             unsigned pend_old = 0, pend_expected = 0;
-            auto settle = [&]() {
+            auto settle = [&](int pending_groups) {
                 if (n >= 2) {
                     int verdict = -1;
                     if (pend_t >= 0 && pend_old + 1 == pend_expected) { fence_acq_rel_gpu(); verdict = pend_t; }
                     s_final[(n - 2) & 7] = verdict;
                 }
                 if (n >= 1) {
-                    asm volatile("cp.async.bulk.wait_group 1;" ::: "memory");
+                    if (pending_groups == 2) asm volatile("cp.async.bulk.wait_group 2;" ::: "memory");
+                    else                     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
                     pend_t = prev_t;
                     if (prev_t >= 0) {
                         pend_expected = CAUSAL ? static_cast<unsigned>(prev_i + 1) : static_cast<unsigned>(prev_Tr);
@@ -404,42 +382,49 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             };
+            // One staging step: panel 0 then panel 1, each handed over by the drain on its own barrier and given back as
+            // soon as the TMA engine has read it, so that the drain writes one panel while the other is being read.
+            auto step = [&](auto issue_panel) -> bool {
+                if (!mbar_wait_relaxed_ool(bar(STG_FULL + 0), n & 1, &abort_flag)) return false;
+                issue_panel(0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                if (!mbar_wait_relaxed_ool(bar(STG_FULL + 1), n & 1, &abort_flag)) return false;
+                issue_panel(1);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");      // panel 0 has been read
+                mbar_arrive(bar(STG_FREE + 0));
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // panel 1 has been read
+                mbar_arrive(bar(STG_FREE + 1));
+                return true;
+            };
             for (int w = 0, e = 0; ok && bwd_item<CAUSAL, GENERAL>(e, prm, item); ++w) {
                 BwdPairPos<GENERAL> pos;
                 for (int it = 0; it < item.nq; ++it, pos.next(item)) {
-                    ok = mbar_wait_relaxed_ool(bar(STG_FULL), n & 1, &abort_flag);
-                    if (!ok) break;
                     const int i = item.i0 + pos.ii;
                     const int qrow = pos.row(item, prm);
-                    tma_reduce_add_2d(&tmAcc, sStg, 0, qrow);                         // columns [0,32)
-                    tma_reduce_add_2d(&tmAcc, sStg + Cfg::TILE_BYTES, 32, qrow);      // columns [32,64)
-                    tma_store_commit_and_wait();                  // staging read; the adds complete asynchronously
-                    mbar_arrive(bar(STG_FREE));
-                    settle();
+                    ok = step([&](int p) { tma_reduce_add_2d(&tmAcc, sStg + p * Cfg::TILE_BYTES, 32 * p, qrow); });   // columns [32 p, 32 p + 32)
+                    if (!ok) break;
+                    settle(2);
                     prev_t = qrow >> 7;
                     prev_i = i;
                     prev_Tr = item.Tr;
                     ++n;
                 }
                 if (!ok) break;
-                ok = mbar_wait_relaxed_ool(bar(STG_FULL), n & 1, &abort_flag);
-                if (!ok) break;
                 const int kvrow0 = item.bh * prm.N + item.j * 128;
-                tma_store_2d(&tmdV, sStg, 0, kvrow0);
-                tma_store_2d(&tmdK, sStg + Cfg::TILE_BYTES, 0, kvrow0);
-                tma_store_commit_and_wait();
-                mbar_arrive(bar(STG_FREE));
-                settle();
+                ok = step([&](int p) { tma_store_2d(p ? &tmdK : &tmdV, sStg + p * Cfg::TILE_BYTES, 0, kvrow0); });
+                if (!ok) break;
+                settle(2);
                 prev_t = -1;
                 ++n;
             }
-            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // everything written before exit
-            if (ok) {                                             // verdicts on the last two steps
-                settle();
+            if (ok) {                                             // everything written before exit; verdicts on the last two steps
+                settle(0);
                 ++n;
                 prev_t = -1;
-                settle();
+                settle(0);
             }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
             mbar_arrive(bar(FIN));
         }
         __syncwarp();
@@ -450,16 +435,21 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         auto finish_tile = [&](int t) { bwd64_finish_tile(prm.dq_acc, prm.dq, prm.scale, t, r); };
         bool ok = true;
         int g = 0, n = 0;
-        // Before writing the staging buffer in step n: the previous TMA must have read it.  The staging consumer
-        // wrote the verdict on step n-4 before that STG_FREE arrival and rewrites the slot only after the STG_FULL
-        // arrivals of later steps: read it here, use it after the stores.
-        auto staging_ready = [&](int& fi) -> bool {
+        if (lane == 0) mbar_arrive(bar(B_READY));                 // "dQ of the pair before the first one has been read"
+        // Before writing staging panel p in step n: the TMA transfer of step n-1 must have read it.
+        auto panel_ready = [&](int p) -> bool {
             bool o = true;
-            if (n > 0) o = mbar_wait_relaxed_ool(bar(STG_FREE), (n - 1) & 1, &abort_flag);
-            o = __all_sync(0xffffffffu, o);
-            fi = (o && n >= 4) ? s_final[(n - 4) & 7] : -1;
-            return o;
+            if (n > 0) o = mbar_wait_relaxed_ool(bar(STG_FREE + p), (n - 1) & 1, &abort_flag);
+            return __all_sync(0xffffffffu, o);
         };
+        auto panel_written = [&](int p) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(STG_FULL + p));
+        };
+        // The staging consumer wrote the verdict on step n-4 before it gave panel 0 of step n-1 back and rewrites the
+        // slot only many steps later: read it once panel 0 is ours.
+        auto verdict = [&]() { return (n >= 4) ? s_final[(n - 4) & 7] : -1; };
         for (int w = 0, e = 0; ok && bwd_item<CAUSAL, GENERAL>(e, prm, item); ++w) {
             for (int it = 0; it < item.nq; ++it, ++g, ++n) {
                 ok = mbar_wait_relaxed_ool(bar(DQ_FULL), g & 1, &abort_flag);
@@ -471,33 +461,38 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tmem_ld32(tmem + Cfg::DQ_COL + lane_base + 32, b);
                 tmem_wait_ld();
                 tc_fence_before();
-                mbar_arrive(bar(DQ_EMPTY));                       // the dQ columns may be overwritten
-                int fi;
-                ok = staging_ready(fi);
-                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(B_READY));         // the dQ columns may be overwritten
                 // two [128 rows][32 floats = 128 bytes] panels, 128-byte swizzle
+                ok = panel_ready(0);
+                if (!ok) break;
+                const int fi = verdict();
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
+                for (int c = 0; c < 8; ++c)
                     *reinterpret_cast<uint4*>(sStg_ptr + r * 128 + ((c ^ (r & 7)) << 4)) =
                         make_uint4(a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
+                panel_written(0);
+                ok = panel_ready(1);
+                if (!ok) break;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
                     *reinterpret_cast<uint4*>(sStg_ptr + Cfg::TILE_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) =
                         make_uint4(b[4 * c], b[4 * c + 1], b[4 * c + 2], b[4 * c + 3]);
-                }
-                fence_proxy_async_smem();
-                mbar_arrive(bar(STG_FULL));
+                panel_written(1);
                 if (fi >= 0) finish_tile(fi);
             }
             if (!ok) break;
             // ---- dV and scale * dK of the item -> BF16 -> staging (dV | dK, [128 rows][64 BF16], 128-byte swizzle)
-            ok = mbar_wait_relaxed_ool(bar(DKV_DONE), w & 1, &abort_flag);
+            ok = mbar_wait_relaxed_ool(bar(B_DONE + ((g - 1) & 1)), ((g - 1) >> 1) & 1, &abort_flag);     // the item's last pair: dV, dK are final
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            int fi;
-            ok = staging_ready(fi);
-            if (!ok) break;
+            int fi = -1;
 #pragma unroll
             for (int t = 0; t < 2; ++t) {                         // t = 0: dV, t = 1: scale * dK
+                ok = panel_ready(t);
+                if (!ok) break;
+                if (t == 0) fi = verdict();
                 const float mul = t ? prm.scale : 1.0f;
                 uint8_t* stage = sStg_ptr + t * Cfg::TILE_BYTES + r * 128;
 #pragma unroll
@@ -516,11 +511,14 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         *reinterpret_cast<uint4*>(stage + ((cc ^ (r & 7)) << 4)) = o;
                     }
                 }
+                if (t == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(DKV_FREE));    // the next item may start new dV, dK accumulators
+                }
+                panel_written(t);
             }
-            tc_fence_before();
-            mbar_arrive(bar(DKV_FREE));                           // the next item may start new dV, dK accumulators
-            fence_proxy_async_smem();
-            mbar_arrive(bar(STG_FULL));
+            if (!ok) break;
             if (fi >= 0) finish_tile(fi);
             ++n;
         }
@@ -544,6 +542,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const float c_l2 = prm.scale * LOG2E;
         bool ok = true;
         int g = 0;
+        if (lane == 0) mbar_arrive(bar(A_READY));                 // "S^T, dP^T of the pair before the first one are free"
         for (int w = 0, e = 0; ok && bwd_item<CAUSAL, GENERAL>(e, prm, item); ++w) {
             int ii = 0;                                           // query tile offset inside the current query head
             for (int it = 0; it < item.nq; ++it, ++g, ii = (GENERAL && ii + 1 == item.nqh) ? 0 : ii + 1) {
@@ -553,10 +552,10 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 uint8_t* xrow = sX_ptr + buf * Cfg::X_BYTES + half * Cfg::TILE_BYTES + r * 128;
-                // the pair on the causal diagonal: key row r sees query column q only if r <= q.  One copy of the arithmetic
-                // for both kinds of pair (instruction-cache footprint); the mask sits behind a CTA-uniform branch.
                 // Partly masked pairs: the causal diagonal (key row r sees query column q only if r <= q), key rows and query
                 // columns beyond the sequence length.  Key row r of the tile sees the query columns q with qlo <= q < qlo + span.
+                // One copy of the arithmetic for both kinds of pair (instruction-cache footprint); the mask sits behind a
+                // CTA-uniform branch.
                 const bool diag = CAUSAL && ii == 0;             // first query tile of a query head
                 const int kvalid = GENERAL ? item.seqlen - item.j * 128 : 128;
                 const int qvalid = GENERAL ? item.seqlen - (item.i0 + ii) * 128 : 128;
@@ -564,7 +563,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int qlo = (GENERAL && r >= kvalid) ? 128 : (diag ? r : 0);
                 const unsigned span = (qvalid > qlo) ? static_cast<unsigned>(qvalid - qlo) : 0u;
                 {
-// not unrolled: the two chunks share one copy of the arithmetic (the unrolled loop body no longer fitted the
+                    // not unrolled: the two chunks share one copy of the arithmetic (the unrolled loop body no longer fitted the
                     // instruction cache next to the other roles' code: 6 % slower)
 #pragma unroll 1
                     for (int h = 0; h < 2; ++h) {
@@ -575,7 +574,8 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         tmem_wait_ld();
                         if (h == 1) {                                 // S^T, dP^T of this pair are in registers: A of the next pair may run
                             tc_fence_before();
-                            mbar_arrive(bar(SDP_FREE));
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar(A_READY + (g + 1) % Cfg::QS));
                         }
                         uint32_t pk[16], dsk[16];
 #pragma unroll
@@ -606,11 +606,10 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             dsk[(c >> 1)] = pack_bf16(ds[0], ds[1]);
                             dsk[(c >> 1) + 1] = pack_bf16(ds[2], ds[3]);
                         }
-                        if (h == 0) {
-                            // first write of this pair into P^T and dS^T: dV of pair g-1 and dK, dQ of pair g-2 must have
-                            // read them (they ran under the arithmetic above)
-                            if (g > 0) ok = mbar_wait_ool(bar(PT_FREE), (g - 1) & 1, &abort_flag);
-                            if (ok && g > 1) ok = mbar_wait_ool(bar(X_FREE + buf), ((g >> 1) - 1) & 1, &abort_flag);
+                        if (h == 0 && g > 0) {
+                            // first write of this pair into P^T and dS^T: dV of pair g-1 (and with it dK, dQ of pair g-2) must
+                            // have read them (they ran under the arithmetic above)
+                            ok = mbar_wait_ool(bar(DQ_FULL), (g - 1) & 1, &abort_flag);
                         }
                         tmem_st16(tmem + Cfg::PT_COL + lane_base + (q0 >> 1), pk);
                         // dS^T row r, 32 queries: four 16-byte chunks of this half's panel, 128-byte swizzle
@@ -627,7 +626,8 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tmem_wait_st();
                 fence_proxy_async_smem();
                 tc_fence_before();
-                mbar_arrive(bar(PDS_FULL + buf));
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(bar(B_READY)); mbar_arrive(bar(PDS_FULL + buf)); }
             }
         }
     }
