@@ -59,6 +59,16 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t par
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
+// Split probe of a barrier: the try_wait is issued at one point of the program and its result is looked at later, so
+// that the shared-memory round trip (200-300 clocks while MMAs run) passes under the arithmetic in between.  The
+// predicate lives in a register declared once at function scope (MBAR_PROBE_DECL at the top of the kernel, outside any
+// loop); NAME must be unique within the kernel.
+#define MBAR_PROBE_DECL(NAME) asm volatile(".reg .pred " #NAME ";")
+#define MBAR_PROBE(NAME, bar, parity) \
+    asm volatile("mbarrier.test_wait.parity.shared::cta.b64 " #NAME ", [%0], %1;" ::"r"(bar), "r"(parity) : "memory")
+#define MBAR_PROBE_SET(NAME, value) asm volatile("setp.ne.b32 " #NAME ", %0, 0;" ::"r"(static_cast<uint32_t>(value)))
+__device__ __forceinline__ bool mbar_probe_result_impl(uint32_t ok) { return ok != 0; }
+#define MBAR_PROBE_RESULT(NAME) ([&]() { uint32_t ok_; asm volatile("selp.u32 %0, 1, 0, " #NAME ";" : "=r"(ok_)); return ok_ != 0; }())
 // Bounded waits.  `abort_flag` is a CTA-shared word: once any role has given up, every later wait returns false
 // soon after.  Returns true when the phase completed.  The abort flag and the clock are looked at once per 1024
 // (256) polls.  Two flavours of each:
