@@ -14,7 +14,6 @@
 #include "bwd_kernel_d128.cuh"
 #include "delta_dp_kernel.cuh"
 #include "fwd_kernel.cuh"
-#include "fwd_kernel_d64.cuh"
 #include "selftest_kernel.cuh"
 
 // Scratch for attn_bwd_static(): lives in the library's device image, so every GPU that loads the
@@ -173,23 +172,6 @@ int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& 
                ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-// d = 64: persistent, one CTA per SM with two query-tile slots
-template <int MODE, bool CAUSAL, bool COUNT, bool PADDED = false>
-int launch_fwd64(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
-                 const attn::FwdParams& prm, cudaStream_t st)
-{
-    using Cfg = attn::Fwd64Cfg;
-    constexpr auto kern = attn::attn_fwd64_kernel<MODE, CAUSAL, COUNT, PADDED>;
-    if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
-    DeviceInfo di;
-    if (int e = device_info(&di)) return e;
-    const long long items = static_cast<long long>(prm.Tr) * prm.BH;
-    const long long want = (items + Cfg::SLOTS - 1) / Cfg::SLOTS;
-    const unsigned grid = static_cast<unsigned>(want < di.sm_count ? want : di.sm_count);
-    return launch_pdl(kern, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tq, tk, tv, to, prm) == cudaSuccess
-               ? ATTN_OK : ATTN_ERR_CUDA;
-}
-
 template <bool CAUSAL, bool GENERAL>
 int launch_bwd_d128(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                     const CUtensorMap& tdk, const CUtensorMap& tdv, const attn::BwdParams& prm, cudaStream_t st)
@@ -277,7 +259,7 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
 
     const long long rows = static_cast<long long>(B) * H * N;
     CUtensorMap tq, tk, tv, to;
-    const int bc = (d == 64) ? attn::Fwd64Cfg::BC : attn::FwdCfg<128>::BC;
+    const int bc = attn::FwdCfg<64>::BC;
     const long long kvrows = static_cast<long long>(B) * Hkv * N;
     if (!make_map(&tq, q, rows, d, 128) || !make_map(&tk, k, kvrows, d, bc) || !make_map(&tv, v, kvrows, d, bc) ||
         !make_map(&to, o, rows, d, 128))
@@ -306,19 +288,17 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     if (!causal && (seqlen % bc != 0 || seqlens)) {
         if (ones) return ATTN_ERR_SHAPE;
         const bool m1 = (mode & ATTN_MODE_STABILISED) != 0;
-        if (d == 64) return m1 ? launch_fwd64<1, false, false, true>(tq, tk, tv, to, prm, st)
-                               : launch_fwd64<0, false, false, true>(tq, tk, tv, to, prm, st);
+        if (d == 64) return m1 ? launch_fwd<64, 1, false, false, true>(tq, tk, tv, to, prm, st)
+                               : launch_fwd<64, 0, false, false, true>(tq, tk, tv, to, prm, st);
         return m1 ? launch_fwd<128, 1, false, false, true>(tq, tk, tv, to, prm, st)
                   : launch_fwd<128, 0, false, false, true>(tq, tk, tv, to, prm, st);
     }
     switch (key) {
-#define FWD64_CASE(K, M_, C_, N_) case K: return launch_fwd64<M_, C_, N_>(tq, tk, tv, to, prm, st);
-        FWD64_CASE(0, 0, false, false)   FWD64_CASE(1, 0, false, true)
-        FWD64_CASE(2, 0, true, false)    FWD64_CASE(3, 0, true, true)
-        FWD64_CASE(4, 1, false, false)   FWD64_CASE(5, 1, false, true)
-        FWD64_CASE(6, 1, true, false)    FWD64_CASE(7, 1, true, true)
-#undef FWD64_CASE
 #define FWD_CASE(K, D_, M_, C_, N_) case K: return launch_fwd<D_, M_, C_, N_>(tq, tk, tv, to, prm, st);
+        FWD_CASE(0, 64, 0, false, false)   FWD_CASE(1, 64, 0, false, true)
+        FWD_CASE(2, 64, 0, true, false)    FWD_CASE(3, 64, 0, true, true)
+        FWD_CASE(4, 64, 1, false, false)   FWD_CASE(5, 64, 1, false, true)
+        FWD_CASE(6, 64, 1, true, false)    FWD_CASE(7, 64, 1, true, true)
         FWD_CASE(8, 128, 0, false, false)  FWD_CASE(9, 128, 0, false, true)
         FWD_CASE(10, 128, 0, true, false)  FWD_CASE(11, 128, 0, true, true)
         FWD_CASE(12, 128, 1, false, false) FWD_CASE(13, 128, 1, false, true)
@@ -575,8 +555,8 @@ int attn_get_tiles(int d, int* Br, int* Bc)
 {
     if (d != 64 && d != 128) return ATTN_ERR_SHAPE;
     if (!Br || !Bc) return ATTN_ERR_NULL;
-    *Br = 128;
-    *Bc = (d == 64) ? attn::Fwd64Cfg::BC : attn::FwdCfg<128>::BC;
+    *Br = attn::FwdCfg<64>::BR;
+    *Bc = attn::FwdCfg<64>::BC;
     return ATTN_OK;
 }
 

@@ -59,16 +59,6 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t par
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-// Split probe of a barrier: the try_wait is issued at one point of the program and its result is looked at later, so
-// that the shared-memory round trip (200-300 clocks while MMAs run) passes under the arithmetic in between.  The
-// predicate lives in a register declared once at function scope (MBAR_PROBE_DECL at the top of the kernel, outside any
-// loop); NAME must be unique within the kernel.
-#define MBAR_PROBE_DECL(NAME) asm volatile(".reg .pred " #NAME ";")
-#define MBAR_PROBE(NAME, bar, parity) \
-    asm volatile("mbarrier.test_wait.parity.shared::cta.b64 " #NAME ", [%0], %1;" ::"r"(bar), "r"(parity) : "memory")
-#define MBAR_PROBE_SET(NAME, value) asm volatile("setp.ne.b32 " #NAME ", %0, 0;" ::"r"(static_cast<uint32_t>(value)))
-__device__ __forceinline__ bool mbar_probe_result_impl(uint32_t ok) { return ok != 0; }
-#define MBAR_PROBE_RESULT(NAME) ([&]() { uint32_t ok_; asm volatile("selp.u32 %0, 1, 0, " #NAME ";" : "=r"(ok_)); return ok_ != 0; }())
 // Bounded waits.  `abort_flag` is a CTA-shared word: once any role has given up, every later wait returns false
 // soon after.  Returns true when the phase completed.  The abort flag and the clock are looked at once per 1024
 // (256) polls.  Two flavours of each:
@@ -181,11 +171,6 @@ __device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, uint32_t src_sm
 __device__ __forceinline__ void tma_store_commit_and_wait() {
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-// Ask L2 for a tile ahead of its load (no shared-memory destination, no completion to wait for).
-__device__ __forceinline__ void tma_prefetch_l2_2d(const void* tmap, int32_t x, int32_t y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");

@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_host_only_entry_points():
-    assert attn.attn_get_tiles(64) == (128, 128)
+    assert attn.attn_get_tiles(64) == (128, 64)
     assert attn.attn_get_tiles(128) == (128, 64)
     with pytest.raises(attn.AttnError) as e:
         attn.attn_get_tiles(96)
