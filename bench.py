@@ -3,11 +3,15 @@
 over one batch of the GPT-2-small-shaped causal workload (B=16, H=12, N=1024, d=64, BF16).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--mode 0|1] [--impl ours|reference]
+                  [--scaling weak|strong] [--context-libs]
 
 Prints one JSON line (rank 0).  Metric: attention fwd+bwd TFLOP/s with the FLOP convention
 fwd 4*Pi*d, bwd 10*Pi*d, Pi = B*H*N^2/2 score pairs for causal attention.
-Multi-GPU: the (batch, head) problems are independent, so every rank runs the same batch
-shape on its own GPU with no data-path collective (weak scaling); time = max over ranks.
+Multi-GPU: the (batch, head) problems are independent, so there is no data-path collective.
+--scaling weak (default): every rank runs the whole batch shape on its own GPU; --scaling strong: one
+batch is split over the ranks by contiguous (batch, head) ranges.  Time = max over ranks.
+--context-libs adds, under its own key, the same workload timed through the attention kernels of
+libraries that ship with the image (library code: context for the reader, not a reference arm).
 """
 import argparse
 import json
@@ -32,8 +36,8 @@ def flops(B, H, N, d, causal):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_bwd_kernel_d64 launch on C2 (ncu capture summarised in
-# profiles/attn_bwd_kernel_d64_C2.md): 211.5 MB + 114.1 MB.
-BWD_DRAM_BYTES_PER_LAUNCH_C2 = 321.6e6
+# profiles/attn_bwd_kernel_d64_C2.md): 209.3 MB + 111.3 MB.
+BWD_DRAM_BYTES_PER_LAUNCH_C2 = 320.6e6
 
 
 def measured_peaks():
@@ -106,11 +110,12 @@ class ClockSampler:
                     samples=len(s))
 
 
-def cpu_baseline(sample_heads, repeat=1):
+def cpu_baseline(sample_heads, repeat=1, workload=WORKLOAD):
     """The oracle as it stands (BF16-emulating forward + delta + backward) timed on the host cores,
-    on `sample_heads` heads of the benchmark workload."""
+    on `sample_heads` heads of `workload`."""
     import attn_inputs as ai
     import oracle
+    WORKLOAD = workload
     H0 = ai.CONFIGS[WORKLOAD][1]
     Bs, Hs = (sample_heads // H0, H0) if sample_heads % H0 == 0 else (1, sample_heads)
     t, m = ai.make(WORKLOAD, B=Bs, H=Hs)
@@ -159,7 +164,11 @@ def run_reference(args):
 
 
 
-def other_workloads(attn, torch, steps=5):
+# heads of C4 / C5 the oracle is timed on (one head of either is 10-20 s of host work)
+CPU_SAMPLE_HEADS = {"C4": 1, "C5": 1}
+
+
+def other_workloads(attn, torch, steps=5, cpu=True):
     """Context lines for the other configurations of the scope table (the headline stays C2): device-timed
     fwd + bwd throughput with inputs resident in HBM, a few steps each.  Inputs are torch-seeded Gaussians of the
     configuration's shape (throughput does not depend on the values); C4 and C5 exceed the L2 by themselves,
@@ -204,6 +213,70 @@ def other_workloads(attn, torch, steps=5):
                                      "ms_per_step": ms, "tflops": (f_fwd + f_bwd) / (ms * 1e-3) / 1e12}
         del sets, o, lse, delta, dq, dk, dv, ws
         torch.cuda.empty_cache()
+        if cpu and name in CPU_SAMPLE_HEADS:
+            out[f"{name}_mode{mode}"]["cpu_baseline"], _ = cpu_baseline(CPU_SAMPLE_HEADS[name], workload=name)
+    return out
+
+
+def context_libs(torch, steps=20):
+    """Library context (not a reference arm, no part of the product path): the headline workload's forward + backward
+    through torch's scaled_dot_product_attention with its cuDNN and flash-attention back ends, on tensors of the same
+    shape.  Each is captured into a CUDA graph (forward + autograd backward) and replayed, so that the time is the
+    device's and not the host's; where capture fails the eager time is given and marked."""
+    import attn_inputs as ai
+    import torch.nn.functional as F
+    from torch.nn.attention import SDPBackend, sdpa_kernel
+    B, H, N, d, causal = ai.CONFIGS[WORKLOAD]
+    f_fwd, f_bwd = flops(B, H, N, d, causal)
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    sets = []
+    for _ in range(N_INPUT_SETS):
+        q, k, v = (torch.randn((B, H, N, d), device="cuda", generator=gen).to(torch.bfloat16).requires_grad_()
+                   for _ in range(3))
+        dO = (0.1 * torch.randn((B, H, N, d), device="cuda", generator=gen)).to(torch.bfloat16)
+        sets.append((q, k, v, dO))
+    out = {}
+    for label, backend in (("torch_sdpa_cudnn", SDPBackend.CUDNN_ATTENTION), ("torch_sdpa_flash", SDPBackend.FLASH_ATTENTION)):
+        try:
+            with sdpa_kernel(backend):
+                def one(x):
+                    q, k, v, dO = x
+                    o = F.scaled_dot_product_attention(q, k, v, is_causal=causal)
+                    return torch.autograd.grad(o, (q, k, v), dO)
+
+                for x in sets:
+                    one(x)
+                torch.cuda.synchronize()
+                how = "cuda graph replay"
+                try:
+                    graphs = []
+                    side = torch.cuda.Stream()
+                    side.wait_stream(torch.cuda.current_stream())
+                    with torch.cuda.stream(side):
+                        for x in sets:
+                            g = torch.cuda.CUDAGraph()
+                            with torch.cuda.graph(g, stream=side):
+                                keep = one(x)
+                            graphs.append((g, keep))
+                    torch.cuda.current_stream().wait_stream(side)
+                    run = lambda i: graphs[i % len(graphs)][0].replay()
+                except Exception:
+                    torch.cuda.synchronize()
+                    how = "eager (graph capture failed: host launch overhead included)"
+                    run = lambda i: one(sets[i % len(sets)])
+                for i in range(3):
+                    run(i)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(steps):
+                    run(i)
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / steps
+                out[label] = {"ms_per_step": ms, "tflops": (f_fwd + f_bwd) / (ms * 1e-3) / 1e12, "how": how}
+        except Exception as e:            # a back end that is not available for this shape on this box
+            out[label] = {"unavailable": str(e).splitlines()[0][:200]}
     return out
 
 def main():
@@ -215,6 +288,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true", help="skip the context lines for C2 mode 1, C4 and C5")
+    ap.add_argument("--scaling", default="weak", choices=("weak", "strong"),
+                    help="weak: the whole batch on every rank; strong: one batch split over the ranks by (batch, head) ranges")
+    ap.add_argument("--context-libs", action="store_true",
+                    help="also time the image's library attention kernels on the same workload (context, printed under its own key)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -236,10 +313,20 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    B, H, N, d, causal = ai.CONFIGS[WORKLOAD]
+    B0, H0, N, d, causal = ai.CONFIGS[WORKLOAD]
     alpha = 1.0 / math.sqrt(d)
     mode = args.mode
-    f_fwd, f_bwd = flops(B, H, N, d, causal)
+    strong = args.scaling == "strong" and world > 1
+    if strong:
+        # one batch for the whole job: this rank owns a contiguous range of its (batch, head) problems and calls the
+        # library on that range as a [1, heads, N, d] problem
+        from paper_2510_04212_b200.sharding import head_slice, shard_view
+        h0, h1 = head_slice(B0 * H0, world, rank)
+        B, H = 1, h1 - h0
+    else:
+        B, H = B0, H0
+    f_fwd, f_bwd = flops(B, H, N, d, causal)                 # this rank's share
+    job_flops = sum(flops(B0, H0, N, d, causal)) * (1 if strong else world)
 
     # ---- inputs: N_INPUT_SETS seeded sets, resident in HBM before any timed region
     def dev_bf16(bits):
@@ -247,7 +334,9 @@ def main():
 
     host_sets, sets = [], []
     for s in range(N_INPUT_SETS):
-        t, _ = ai.make(WORKLOAD, seed=ai.SEEDS[WORKLOAD] + 1000 * s + 17 * rank)
+        t, _ = ai.make(WORKLOAD, seed=ai.SEEDS[WORKLOAD] + 1000 * s + (0 if strong else 17 * rank))
+        if strong:
+            t = {n: shard_view(t[n], B0, H0, world, rank) for n in ("q", "k", "v", "dO")}
         host = {n: torch.from_numpy(np.ascontiguousarray(t[n]).view(np.int16)).view(torch.bfloat16).pin_memory()
                 for n in ("q", "k", "v", "dO")}
         host_sets.append(host)
@@ -294,6 +383,31 @@ def main():
         e1.record()
         barrier()
         ms_total = e0.elapsed_time(e1)
+
+        # ---- region A2: the same rotated steps, one event pair per step: the distribution of the step time (an event
+        # between two steps keeps the next forward's prologue from overlapping the previous kernel's tail, so these
+        # are a little longer than the mean of region A)
+        n_each = max(20, args.steps)
+        pe = [torch.cuda.Event(enable_timing=True) for _ in range(n_each + 1)]
+        pe[0].record()
+        for k in range(n_each):
+            step(sets[k % N_INPUT_SETS])
+            pe[k + 1].record()
+        torch.cuda.synchronize()
+        each = sorted(pe[k].elapsed_time(pe[k + 1]) for k in range(n_each))
+
+        # ---- region A3: the same number of steps on ONE input set (its 101 MB of inputs and the outputs of the
+        # previous step stay in the 126 MB L2 as far as they fit): the unflushed figure
+        for w in range(3):
+            step(sets[0])
+        barrier()
+        u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        u0.record()
+        for k in range(args.steps):
+            step(sets[0])
+        u1.record()
+        barrier()
+        ms_single_set = u0.elapsed_time(u1) / args.steps
 
         # ---- region B: the same K steps with events between the kernels (per-kernel durations)
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
@@ -386,49 +500,71 @@ def main():
     if attn.attn_last_device_status() != 0:
         raise SystemExit("device-side wait timed out during the timed region")
 
+    ms_median = each[len(each) // 2]
     if dist is not None:
-        tt = torch.tensor([ms_total, ms_e2e], device="cuda", dtype=torch.float64)
+        tt = torch.tensor([ms_total, ms_e2e, ms_median, ms_single_set], device="cuda", dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(tt[0]), float(tt[1])
+        ms_total, ms_e2e, ms_median, ms_single_set = (float(x) for x in tt)
     ms_step = ms_total / args.steps
-    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
-    e2e_value = world * (f_fwd + f_bwd) / (ms_e2e * 1e-3) / 1e12
+    value = job_flops / (ms_step * 1e-3) / 1e12
+    e2e_value = job_flops / (ms_e2e * 1e-3) / 1e12
     elem_bytes = B * H * N * d * 2
 
     if rank == 0:
         peaks = measured_peaks()
         bwd_ms = per_kernel[2]
         achieved = f_bwd / (bwd_ms * 1e-3) / 1e12
+        clk = clocks.summary()
+        # forward at d = 64: the exponentials bind before the tensor pipe does.  One ex2 per score pair that counts
+        # (Pi = B*H*N^2/2), against 16 ex2 per clock per SM (4 per SM sub-partition) x 148 SMs x the SM clock
+        # sampled during the timed regions.
+        sm_mhz = clk["sm_mhz"] or clk["sm_max_mhz"] or 1965
+        pairs = B * H * N * N * (0.5 if causal else 1.0)
+        mufu_peak = 16 * 148 * sm_mhz * 1e6 / 1e9            # Gex2/s
+        mufu_achieved = pairs / (per_kernel[0] * 1e-3) / 1e9
         out = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong" if strong else "weak",
+            "ms_per_step_each": {"n": len(each), "median": ms_median, "min": each[0], "p90": each[(9 * len(each)) // 10],
+                                 "max": each[-1], "how": "one CUDA-event pair per step, rotated input sets"},
+            "ms_per_step_single_set": ms_single_set,
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{WORKLOAD}: B={B},H={H},N={N},d={d},causal, mode={mode} (per GPU)",
+            "config": {"workload": (f"{WORKLOAD}: B={B0},H={H0},N={N},d={d},causal, mode={mode} "
+                                    + (f"(one batch split over {world} GPUs, {H} of {B0 * H0} heads on rank 0)" if strong
+                                       else "(per GPU)")),
                        "l2": f"{N_INPUT_SETS} input sets rotated ({N_INPUT_SETS * 4 * elem_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "flop_convention": "fwd 4*Pi*d + bwd 10*Pi*d, Pi=B*H*N^2/2"},
             "frac_of_bf16_peak": value / world / peaks["bf16_tflops"],
             "frac_of_nominal_2250": value / world / 2250.0,
+            "frac_of_bf16_peak_median_step": (f_fwd + f_bwd) / (ms_median * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "kernels_ms": {"attn_fwd_kernel": per_kernel[0], "bwd_preprocess_kernel": per_kernel[1],
                            "attn_bwd_kernel": per_kernel[2],
                            "dq_convert_tiled128_kernel": per_kernel[3] if d != 64 else None},
             "fwd_tflops": f_fwd / (per_kernel[0] * 1e-3) / 1e12,
             "delta_pass_gbs": (2 * elem_bytes + 4 * B * H * N) / (per_kernel[1] * 1e-3) / 1e9,
+            "roofline_fwd": {"bound": "mufu", "kernel": "attn_fwd_kernel", "achieved": mufu_achieved, "peak": mufu_peak,
+                             "unit": "Gex2/s", "frac": mufu_achieved / mufu_peak,
+                             "peak_source": f"16 ex2/clk/SM x 148 SMs x {sm_mhz} MHz (median SM clock sampled in the timed regions)",
+                             "tensor_frac": f_fwd / (per_kernel[0] * 1e-3) / 1e12 / peaks["bf16_tflops"]},
             "roofline": {"bound": "tensor", "kernel": "attn_bwd_kernel", "achieved": achieved,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                          "peak_source": peaks["source"] + " (burst)",
-                         "traffic": BWD_DRAM_BYTES_PER_LAUNCH_C2 if WORKLOAD == "C2" else None,
+                         "traffic": BWD_DRAM_BYTES_PER_LAUNCH_C2 if (WORKLOAD == "C2" and not strong) else None,
                          "traffic_unit": "bytes per launch (ncu dram read + write, profiles/attn_bwd_kernel_d64_C2.md)"},
             "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": 4 * elem_bytes,
                     "d2h_bytes_per_step": 4 * elem_bytes + 4 * B * H * N, "ms_per_step": ms_e2e,
                     "how": "pipelined: H2D of step k+1 and D2H of step k on two copy streams around the compute stream, inputs and results double-buffered on the device",
                     "ms_per_step_serial": ms_e2e_serial},
             "gpu_launches": (3 if d == 64 else 4) * args.steps,   # d = 64: the main kernel also finishes dQ
-            "clocks": clocks.summary(),
+            "clocks": clk,
         }
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"], _ = cpu_baseline(96)
         if world == 1 and not args.no_other_workloads:
-            out["other_workloads"] = other_workloads(attn, torch)
+            out["other_workloads"] = other_workloads(attn, torch, cpu=not args.no_cpu_baseline)
+        if world == 1 and args.context_libs:
+            out["context_libs"] = context_libs(torch)
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
