@@ -127,6 +127,28 @@ int attn_fwd_count_ones(const void* q, const void* k, const void* v, void* o, fl
                         void* stream);
 
 /*
+ * attn_fwd plus the output in FP32, for the paper's "O kept in FP32" experiments (Sec. 3.2: the failure goes away
+ * when delta is formed from an O that was not rounded to BF16):
+ *   out: o_f32   FP32 [B][H][N][d], device memory, 16-byte aligned, overwritten: O-bar / l, where O-bar is the FP32
+ *                accumulator of Algorithm 1 / 3 before either of its BF16 roundings and the division is IEEE
+ *                round-to-nearest.  P-bar is still the BF16-rounded matrix (that rounding is the method's).
+ * o and lse are written as by attn_fwd, bit for bit.  A separate kernel instantiation (that of
+ * attn_fwd_count_ones), so attn_fwd does not pay for it.  Errors as attn_fwd; o_f32 == NULL: ATTN_ERR_NULL.
+ * attn_bwd_delta_f32 turns o_f32 into the delta that attn_bwd takes with ATTN_MODE_FLAG_DELTA_GIVEN.
+ */
+int attn_fwd_o_f32(const void* q, const void* k, const void* v, void* o, float* lse, float* o_f32,
+                   int B, int H, int N, int d, int causal, float scale, int mode,
+                   void* stream);
+
+/*
+ * delta = rowsum(dO o O) with O in FP32 (Algorithm 2's first line, on the output of attn_fwd_o_f32; Sec. 3.2):
+ *   in : o_f32  FP32 [B][H][N][d];  dO  BF16 [B][H][N][d]        (device memory, 16-byte aligned)
+ *   out: delta  FP32 [B][H][N]      products and sums in FP32, one rounding per fused multiply-add
+ * Errors: ATTN_ERR_NULL, ATTN_ERR_SHAPE, ATTN_ERR_ALIGN, ATTN_ERR_DEVICE, ATTN_ERR_CUDA.
+ */
+int attn_bwd_delta_f32(const float* o_f32, const void* dO, float* delta, int B, int H, int N, int d, void* stream);
+
+/*
  * attn_fwd_count_ones with P-bar rounded to an 8-bit floating-point format instead of BF16: a diagnostic for the
  * question the paper leaves open (Sec. 5 names FP8 training as future work), not part of its method.
  *   pbar_format  ATTN_PBAR_BF16 (0): exactly attn_fwd_count_ones;
@@ -157,8 +179,11 @@ int attn_bwd_preprocess(const void* o, const void* dO, float* delta,
  * delta = rowsum(dP o P) with dP = dO V^T and P = exp(scale Q K^T - L): the alternative formulation of Sec. 3.2,
  * mathematically the same number as rowsum(dO o O) but computed without O (the paper uses it to show that the
  * error of the BF16 O is what breaks training).  S and dP are FP32 sums of the exact BF16 products, P is not
- * rounded, the row sum is FP32.  A diagnostic on the ordinary FP32 pipes (about a millisecond on the benchmark
- * workload), not a step of the hot path: pass its result to attn_bwd with ATTN_MODE_FLAG_DELTA_GIVEN.
+ * rounded, the row sum is FP32.  A diagnostic, not a step of the hot path, and deliberately slow: it runs the two
+ * contractions on the ordinary FP32 pipes so that every product is exact and every sum a plain FP32 sum in a fixed
+ * order (1.45 ms on B=16, H=12, N=1024, d=64 causal, six times the forward + backward step).  Pass its result to
+ * attn_bwd with ATTN_MODE_FLAG_DELTA_GIVEN.  The cheaper route to a delta free of the rounding of O is
+ * attn_fwd_o_f32 followed by attn_bwd_delta_f32.
  *   in : q, k, v, dO  BF16 [B][H][N][d];  lse FP32 [B][H][N] as written by attn_fwd
  *   out: delta        FP32 [B][H][N]
  * Same shape, scale, alignment and device checks and error codes as attn_fwd; asynchronous on `stream`.

@@ -13,12 +13,12 @@ import os
 
 from . import build as _build
 
-__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
+__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
            "attn_get_tiles", "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout",
            "attn_strerror", "lib", "LIB_PATH", "EXPORTS"]
 
 LIB_PATH = _build.LIB
-EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
+EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
            "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout", "attn_strerror")
 
 
@@ -44,6 +44,10 @@ def _load():
     L.attn_fwd_pbar_format.argtypes = [vp, vp, vp, vp, fp, vp, i, i, i, i, i, f, i, i, vp]
     L.attn_bwd_delta_dp.restype = i
     L.attn_bwd_delta_dp.argtypes = [vp, vp, vp, vp, fp, fp, i, i, i, i, i, C.c_float, vp]
+    L.attn_fwd_o_f32.restype = i
+    L.attn_fwd_o_f32.argtypes = [vp, vp, vp, vp, fp, fp, i, i, i, i, i, f, i, vp]
+    L.attn_bwd_delta_f32.restype = i
+    L.attn_bwd_delta_f32.argtypes = [fp, vp, fp, i, i, i, i, vp]
     L.attn_bwd_preprocess.restype = i
     L.attn_bwd_preprocess.argtypes = [vp, vp, fp, i, i, i, i, vp]
     L.attn_bwd.restype = i
@@ -133,6 +137,16 @@ def attn_fwd_pbar_format(q, k, v, o, lse, ones, B, H, N, d, causal, scale, mode,
 def attn_bwd_delta_dp(q, k, v, dO, lse, delta, B, H, N, d, causal, scale, stream=None):
     _check(lib.attn_bwd_delta_dp(_ptr(q), _ptr(k), _ptr(v), _ptr(dO), _ptr(lse), _ptr(delta), B, H, N, d,
                                  int(bool(causal)), float(scale), _stream(stream)), "attn_bwd_delta_dp")
+
+
+def attn_fwd_o_f32(q, k, v, o, lse, o_f32, B, H, N, d, causal, scale, mode, stream=None):
+    _check(lib.attn_fwd_o_f32(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(o_f32), B, H, N, d,
+                              int(bool(causal)), float(scale), int(mode), _stream(stream)), "attn_fwd_o_f32")
+
+
+def attn_bwd_delta_f32(o_f32, dO, delta, B, H, N, d, stream=None):
+    _check(lib.attn_bwd_delta_f32(_ptr(o_f32), _ptr(dO), _ptr(delta), B, H, N, d, _stream(stream)),
+           "attn_bwd_delta_f32")
 
 
 def attn_bwd_preprocess(o, dO, delta, B, H, N, d, stream=None):

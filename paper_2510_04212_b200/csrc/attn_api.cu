@@ -242,7 +242,7 @@ extern "C" {
 // attn_fwd and attn_fwd_count_ones: `ones` == nullptr selects the instantiations without the counter
 static int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int* ones,
                     int B, int H, int Hkv, int N, int seqlen, const int* seqlens, int d, int causal, float scale, int mode,
-                    void* stream, int pbar_fmt = ATTN_PBAR_BF16)
+                    void* stream, int pbar_fmt = ATTN_PBAR_BF16, float* o_f32 = nullptr)
 {
     if (pbar_fmt != ATTN_PBAR_BF16 && pbar_fmt != ATTN_PBAR_E4M3 && pbar_fmt != ATTN_PBAR_E5M2) return ATTN_ERR_MODE;
     if (!q || !k || !v || !o || !lse) return ATTN_ERR_NULL;
@@ -268,6 +268,7 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     attn::FwdParams prm;
     prm.lse = lse;
     prm.ones = ones;
+    prm.o_f32 = o_f32;
     prm.pbar_fmt = pbar_fmt;
     prm.single_rounding = (mode & ATTN_MODE_FLAG_SINGLE_ROUNDING) ? 1 : 0;
     prm.N = N;
@@ -283,10 +284,10 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     prm.guard_cap = (mode & ATTN_MODE_FLAG_GUARDED) ? g_guard_cap.load() : 0.0f;
     prm.status = status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int key = (d == 128 ? 8 : 0) | ((mode & ATTN_MODE_STABILISED) ? 4 : 0) | (causal ? 2 : 0) | (ones ? 1 : 0);
+    const int key = (d == 128 ? 8 : 0) | ((mode & ATTN_MODE_STABILISED) ? 4 : 0) | (causal ? 2 : 0) | ((ones || o_f32) ? 1 : 0);
     // full attention over a sequence that ends inside a 64-key tile: the instantiations that mask the rest of that tile
     if (!causal && (seqlen % bc != 0 || seqlens)) {
-        if (ones) return ATTN_ERR_SHAPE;
+        if (ones || o_f32) return ATTN_ERR_SHAPE;
         const bool m1 = (mode & ATTN_MODE_STABILISED) != 0;
         if (d == 64) return m1 ? launch_fwd<64, 1, false, false, true>(tq, tk, tv, to, prm, st)
                                : launch_fwd<64, 0, false, false, true>(tq, tk, tv, to, prm, st);
@@ -326,6 +327,30 @@ int attn_fwd_pbar_format(const void* q, const void* k, const void* v, void* o, f
 {
     if (!ones) return ATTN_ERR_NULL;
     return fwd_impl(q, k, v, o, lse, ones, B, H, H, N, N, nullptr, d, causal, scale, mode, stream, pbar_format);
+}
+
+int attn_fwd_o_f32(const void* q, const void* k, const void* v, void* o, float* lse, float* o_f32,
+                   int B, int H, int N, int d, int causal, float scale, int mode, void* stream)
+{
+    if (!o_f32) return ATTN_ERR_NULL;
+    if (!aligned16(o_f32)) return ATTN_ERR_ALIGN;
+    return fwd_impl(q, k, v, o, lse, nullptr, B, H, H, N, N, nullptr, d, causal, scale, mode, stream, ATTN_PBAR_BF16, o_f32);
+}
+
+int attn_bwd_delta_f32(const float* o_f32, const void* dO, float* delta, int B, int H, int N, int d, void* stream)
+{
+    if (!o_f32 || !dO || !delta) return ATTN_ERR_NULL;
+    if (int e = check_shape(B, H, N, d)) return e;
+    if (!aligned16(o_f32) || !aligned16(dO)) return ATTN_ERR_ALIGN;
+    if (int e = check_device()) return e;
+    const long long n_chunks = static_cast<long long>(B) * H * N * (d / 8);
+    const unsigned blocks = static_cast<unsigned>((n_chunks + 255) / 256);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (d == 64)
+        attn::delta_f32_kernel<64><<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(o_f32), static_cast<const uint4*>(dO), delta, n_chunks);
+    else
+        attn::delta_f32_kernel<128><<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(o_f32), static_cast<const uint4*>(dO), delta, n_chunks);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
 int attn_bwd_preprocess(const void* o, const void* dO, float* delta, int B, int H, int N, int d, void* stream)

@@ -67,6 +67,32 @@ bwd_preprocess_kernel(const uint4* __restrict__ o, const uint4* __restrict__ dO,
     }
 }
 
+// ------------------------------------------------------------------ delta = rowsum(dO o O) with O in FP32
+// The "O kept in FP32" variant of Sec. 3.2: same pass, O read as FP32 (the forward's o_f32 output).
+template <int D>
+__global__ void __launch_bounds__(256)
+delta_f32_kernel(const float4* __restrict__ o, const uint4* __restrict__ dO, float* __restrict__ delta, long long n_chunks)
+{
+    constexpr int TPR = D / 8;
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    float acc = 0.0f;
+    if (idx < n_chunks) {
+        const float4 a0 = o[2 * idx], a1 = o[2 * idx + 1];
+        const uint4 b = __ldg(dO + idx);
+        acc = fmaf(a0.x, ptx::bf16_lo(b.x), acc);
+        acc = fmaf(a0.y, ptx::bf16_hi(b.x), acc);
+        acc = fmaf(a0.z, ptx::bf16_lo(b.y), acc);
+        acc = fmaf(a0.w, ptx::bf16_hi(b.y), acc);
+        acc = fmaf(a1.x, ptx::bf16_lo(b.z), acc);
+        acc = fmaf(a1.y, ptx::bf16_hi(b.z), acc);
+        acc = fmaf(a1.z, ptx::bf16_lo(b.w), acc);
+        acc = fmaf(a1.w, ptx::bf16_hi(b.w), acc);
+    }
+#pragma unroll
+    for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (idx < n_chunks && (threadIdx.x % TPR) == 0) delta[idx / TPR] = acc;
+}
+
 // ------------------------------------------------------------------ dQ = bf16(scale * acc), d = 128
 // (at d = 64 the main kernel converts a dQ tile itself when its last contribution has arrived)
 // The d = 128 main kernel's accumulator keeps the layout of that kernel's staging buffer so that a staged panel is

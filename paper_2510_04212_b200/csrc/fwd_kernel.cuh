@@ -65,7 +65,8 @@ struct FwdCfg {
 
 struct FwdParams {
     float* lse;
-    int* ones;                 // COUNT instantiations only: per-row count of P-bar entries equal to 1
+    int* ones;                 // COUNT instantiations only: per-row count of P-bar entries equal to 1 (may be nullptr)
+    float* o_f32;              // COUNT instantiations only, may be nullptr: O = O-bar / l with O-bar left in FP32
     int pbar_fmt;              // COUNT instantiations only: 0 = BF16 P-bar, 1 = E4M3, 2 = E5M2 (diagnostic)
     int single_rounding;       // != 0: O-bar is not rounded to BF16 before the division (diagnostic variant)
     int N, BH, Tr;             // N: rows per head in memory; Tr: 128-row query tiles that hold one of the seqlen queries
@@ -538,6 +539,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 uint32_t r[32];
                 tmem_ld32(tO + c0, r);
                 tmem_wait_ld();
+                if constexpr (COUNT) {
+                    if (prm.o_f32) {                              // the output that skips both BF16 roundings (Sec. 3.2)
+                        float4* dst = reinterpret_cast<float4*>(prm.o_f32 + (static_cast<size_t>(row0) + row) * D + c0);
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            dst[c >> 2] = make_float4(__fdiv_rn(__uint_as_float(r[c]), l), __fdiv_rn(__uint_as_float(r[c + 1]), l),
+                                                      __fdiv_rn(__uint_as_float(r[c + 2]), l), __fdiv_rn(__uint_as_float(r[c + 3]), l));
+                    }
+                }
                 uint32_t out[16];
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
@@ -557,7 +567,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 }
             }
             prm.lse[static_cast<size_t>(row0) + row] = m + lg2(l) * LN2;
-            if (COUNT) prm.ones[static_cast<size_t>(row0) + row] = n_ones;
+            if (COUNT && prm.ones) prm.ones[static_cast<size_t>(row0) + row] = n_ones;
             fence_proxy_async_smem();
             mbar_arrive(bar(EPI));
             if (tid == 0) {

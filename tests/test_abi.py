@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared_symbols():
     text = open(os.path.join(ROOT, "include", "attn.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(attn_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(attn_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
@@ -87,6 +87,11 @@ def test_argument_validation_comes_before_any_device_work():
     assert lib.attn_bwd_delta_dp(None, p, p, p, p, p, 1, 1, 128, 64, 1, 0.125, None) == -1
     assert lib.attn_bwd_delta_dp(p, p, p, p, p, p, 1, 1, 100, 64, 1, 0.125, None) == -2
     assert lib.attn_bwd_delta_dp(p, p, p, p, p, p, 1, 1, 128, 64, 1, -1.0, None) == -4
+    assert lib.attn_fwd_o_f32(p, p, p, p, p, None, 1, 1, 128, 64, 1, 0.125, 0, None) == -1
+    assert lib.attn_fwd_o_f32(p, p, p, p, p, p + 4, 1, 1, 128, 64, 1, 0.125, 0, None) == -9
+    assert lib.attn_fwd_o_f32(p, p, p, p, p, p, 1, 1, 100, 64, 1, 0.125, 0, None) == -2
+    assert lib.attn_bwd_delta_f32(None, p, p, 1, 1, 128, 64, None) == -1
+    assert lib.attn_bwd_delta_f32(p, p, p, 1, 1, 128, 96, None) == -2
     assert lib.attn_bwd_preprocess(None, p, p, 1, 1, 128, 64, None) == -1
     assert lib.attn_bwd_preprocess(p, p, p, 1, 1, 128, 32, None) == -2
 

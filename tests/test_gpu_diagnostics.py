@@ -113,6 +113,60 @@ def test_backward_with_a_given_high_precision_delta(B, H, N, d, causal):
         assert max_abs(got, ref) <= 2e-2 and rel_fro(got, ref) <= 1e-2, n
 
 
+@pytest.mark.parametrize("B,H,N,d,causal,mode", [(1, 2, 384, 64, True, 0), (2, 1, 256, 128, False, 0),
+                                                  (1, 1, 256, 128, True, 1), (1, 2, 256, 64, False, 1)])
+def test_forward_output_in_fp32_and_the_delta_formed_from_it(B, H, N, d, causal, mode):
+    """attn_fwd_o_f32 (Sec. 3.2, O kept in FP32): o and lse as attn_fwd bit for bit; o_f32 against O-bar / l of the emulating
+    oracle (O-bar before its rounding) and closer to the fp64 O than the BF16 output is; attn_bwd_delta_f32 of it
+    against the fp64 row sums, then used as the given delta of the backward pass."""
+    gu, attn = _env()
+    t = ai.gaussian(B, H, N, d, seed=450 + N + d + mode)
+    m = dict(B=B, H=H, N=N, d=d, causal=causal, alpha=d ** -0.5)
+    dev, o0, lse0 = gu.run_fwd(t, m, mode)
+    o = torch.empty_like(o0)
+    lse = torch.empty_like(lse0)
+    o32 = torch.full((B, H, N, d), float("nan"), dtype=torch.float32, device="cuda")
+    attn.attn_fwd_o_f32(dev["q"], dev["k"], dev["v"], o, lse, o32, B, H, N, d, causal, m["alpha"], mode)
+    torch.cuda.synchronize()
+    assert attn.attn_last_device_status() == 0
+    assert np.array_equal(gu.to_bits(o), gu.to_bits(o0)) and np.array_equal(lse.cpu().numpy(), lse0.cpu().numpy())
+    got = o32.cpu().numpy()
+    _, _, dg = oracle.emu_fwd(t["q"], t["k"], t["v"], causal, m["alpha"], mode, diagnostics=True, **_tiles(attn, d))
+    want = dg["obar_f32"] / dg["l"][..., None]                    # float32 / float32: IEEE, as the kernel divides
+    Oref, Lref = oracle.ref_fwd(t["q"], t["k"], t["v"], causal, m["alpha"])
+    # Against the oracle: FP32 accumulation in another order (a few 1e-7 of the condition scale sum_j P_j |V_j| of the
+    # dot product), and now and then a P-bar entry that lands on the other side of a BF16 boundary (one BF16 ulp of one
+    # of the row's weights: at most 2^-8 of that scale, and rare)
+    absv = (t["v"] & np.uint16(0x7FFF)).astype(np.uint16)
+    cond, _ = oracle.ref_fwd(t["q"], t["k"], absv, causal, m["alpha"])
+    diff = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    assert np.all(diff <= 2.0 ** -8 * cond + 1e-30)
+    assert np.mean(diff <= 4e-6 * cond + 1e-30) >= 0.98, np.mean(diff <= 4e-6 * cond + 1e-30)
+    err32 = np.linalg.norm((got.astype(np.float64) - Oref).ravel())
+    err16 = np.linalg.norm((as_f64(gu.to_bits(o)) - Oref).ravel())
+    assert err32 < 0.6 * err16, (err32, err16)                   # the BF16 rounding of O is what it leaves out
+
+    delta = torch.full((B, H, N), float("nan"), dtype=torch.float32, device="cuda")
+    attn.attn_bwd_delta_f32(o32, dev["dO"], delta, B, H, N, d)
+    torch.cuda.synchronize()
+    d_got = delta.cpu().numpy()
+    d_want = (as_f64(t["dO"]) * got.astype(np.float64)).sum(-1)
+    bound = 1e-5 * (np.abs(as_f64(t["dO"])) * np.abs(got.astype(np.float64))).sum(-1) + 1e-30
+    assert np.all(np.abs(d_got - d_want) <= bound)
+    dq, dk, dv = (torch.empty_like(dev["q"]) for _ in range(3))
+    nbytes = attn.attn_bwd_workspace_bytes(B, H, N, d)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    attn.attn_bwd(dev["q"], dev["k"], dev["v"], o, dev["dO"], lse, dq, dk, dv, delta, ws, nbytes,
+                  B, H, N, d, causal, m["alpha"], DELTA_GIVEN)
+    torch.cuda.synchronize()
+    assert attn.attn_last_device_status() == 0
+    dqe, dke, dve = oracle.emu_bwd(t["q"], t["k"], t["v"], t["dO"], lse.cpu().numpy(), d_got, causal, m["alpha"])
+    for g_, e_, n in ((dq, dqe, "dQ"), (dk, dke, "dK"), (dv, dve, "dV")):
+        g_ = gu.to_bits(g_)
+        denom = np.linalg.norm(as_f64(e_).ravel())
+        assert np.linalg.norm((as_f64(g_) - as_f64(e_)).ravel()) <= 2e-3 * denom + 1e-6, n
+
+
 @pytest.mark.parametrize("B,H,N,d,causal", [(1, 2, 384, 64, True), (2, 1, 256, 128, False), (1, 1, 256, 128, True)])
 def test_delta_from_dp_and_p(B, H, N, d, causal):
     """attn_bwd_delta_dp against the fp64 oracle of the same formula (given the same L), and the point of the variant:
