@@ -122,6 +122,10 @@ __device__ __forceinline__ bool bwd_item(int& e, const BwdParams& prm, BwdItem& 
 __device__ __noinline__ void bwd64_finish_tile(const float* dq_acc, uint16_t* dq, float sc, int t, int r)
 {
     constexpr int D = 64;
+    // The tile was written by bulk reduce-adds (async proxy) of this and other CTAs, each complete (bulk-group wait)
+    // before its CTA's releasing increment of the arrival counter, which this CTA's counting thread has acquired.
+    // The reads below go through the generic proxy: order them after the other proxy's writes explicitly.
+    asm volatile("fence.proxy.async.global;" ::: "memory");
     const float4* src = reinterpret_cast<const float4*>(dq_acc + static_cast<size_t>(t) * 128 * D);
     uint4* dst = reinterpret_cast<uint4*>(dq + static_cast<size_t>(t) * 128 * D);
 #pragma unroll
