@@ -322,6 +322,39 @@ int attn_bwd_varlen(const void* q, const void* k, const void* v, const void* o, 
                     const int* seqlens, int B, int H, int H_kv, int N, int d, int causal, float scale, int mode,
                     void* stream);
 
+/*
+ * Packed variable-length batches: B sequences stored one after the other with no padding rows, addressed by
+ * cumulative offsets (the layout training frameworks use for batches of documents of different lengths; the paper's
+ * experiments use a fixed context of 1024, nothing in its method depends on that).
+ *   cu_seqlens  int32 [B + 1], DEVICE memory: sequence b occupies tokens [cu_seqlens[b], cu_seqlens[b + 1]);
+ *               cu_seqlens[0] = 0, non-decreasing, cu_seqlens[B] = T.  A length of 0 is allowed (nothing is written
+ *               for that sequence); a length above N_max is the caller's error (the tokens beyond N_max are ignored).
+ *   q, o, dO, dq   BF16 [T][H][d]      (token-major: the heads of a token are contiguous)
+ *   k, v, dk, dv   BF16 [T][H_kv][d]
+ *   lse, delta     FP32 [H][T]
+ *   T           total number of tokens;  N_max: a multiple of 128, >= every sequence length (it sizes the workspace)
+ * The result for sequence b is that of attn_fwd / attn_bwd (attn_fwd_gqa / attn_bwd_gqa when H_kv < H) on that
+ * sequence alone, with the same tiles, modes and flags; every output row of every token is written, nothing else is.
+ * How: a layout adapter around the per-batch-length kernels (attn_fwd_varlen / attn_bwd_varlen).  The call copies the
+ * packed inputs into padded [B][H][N_max][d] tensors inside `workspace` (streaming kernels, zeros in the unused rows
+ * of partly used tiles), runs those kernels, which skip the tiles that hold only padding, and copies the results
+ * back; all on `stream`, no synchronisation.  The copies move every tensor once more each way (about 8 x the size
+ * of q for a forward + backward); the attention kernels themselves do no work on padding tiles.
+ *   workspace   device memory, 256-byte aligned, at least attn_packed_workspace_bytes(B, H, H_kv, N_max, d, backward)
+ *               bytes (backward = 0 for attn_fwd_packed, 1 for attn_bwd_packed); contents undefined on entry and on
+ *               return.  Too small, NULL or misaligned: ATTN_ERR_WORKSPACE.
+ * With ATTN_MODE_FLAG_DELTA_GIVEN, delta is an input in the packed layout.  Other errors as attn_fwd_varlen /
+ * attn_bwd_varlen; cu_seqlens == NULL: ATTN_ERR_NULL; T < 1 or T * H >= 2^31: ATTN_ERR_SHAPE.
+ */
+size_t attn_packed_workspace_bytes(int B, int H, int H_kv, int N_max, int d, int backward);
+int attn_fwd_packed(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens,
+                    void* workspace, size_t workspace_bytes, int B, int H, int H_kv, int T, int N_max, int d,
+                    int causal, float scale, int mode, void* stream);
+int attn_bwd_packed(const void* q, const void* k, const void* v, const void* o, const void* dO, const float* lse,
+                    void* dq, void* dk, void* dv, float* delta, const int* cu_seqlens,
+                    void* workspace, size_t workspace_bytes, int B, int H, int H_kv, int T, int N_max, int d,
+                    int causal, float scale, int mode, void* stream);
+
 /* Bytes of scratch attn_bwd needs for this shape; 0 if the shape is unsupported. */
 size_t attn_bwd_workspace_bytes(int B, int H, int N, int d);
 

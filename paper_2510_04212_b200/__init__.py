@@ -13,12 +13,12 @@ import os
 
 from . import build as _build
 
-__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
+__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
            "attn_get_tiles", "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout",
            "attn_strerror", "lib", "LIB_PATH", "EXPORTS"]
 
 LIB_PATH = _build.LIB
-EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
+EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
            "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout", "attn_strerror")
 
 
@@ -48,6 +48,12 @@ def _load():
     L.attn_fwd_o_f32.argtypes = [vp, vp, vp, vp, fp, fp, i, i, i, i, i, f, i, vp]
     L.attn_bwd_delta_f32.restype = i
     L.attn_bwd_delta_f32.argtypes = [fp, vp, fp, i, i, i, i, vp]
+    L.attn_packed_workspace_bytes.restype = sz
+    L.attn_packed_workspace_bytes.argtypes = [i, i, i, i, i, i]
+    L.attn_fwd_packed.restype = i
+    L.attn_fwd_packed.argtypes = [vp, vp, vp, vp, fp, vp, vp, sz, i, i, i, i, i, i, i, f, i, vp]
+    L.attn_bwd_packed.restype = i
+    L.attn_bwd_packed.argtypes = [vp, vp, vp, vp, vp, fp, vp, vp, vp, fp, vp, vp, sz, i, i, i, i, i, i, i, f, i, vp]
     L.attn_bwd_preprocess.restype = i
     L.attn_bwd_preprocess.argtypes = [vp, vp, fp, i, i, i, i, vp]
     L.attn_bwd.restype = i
@@ -212,6 +218,24 @@ def attn_bwd_varlen(q, k, v, o, dO, lse, dq, dk, dv, delta, workspace, workspace
     _check(lib.attn_bwd_varlen(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(dO), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv),
                                _ptr(delta), _ptr(workspace), int(workspace_bytes), _ptr(seqlens), B, H, H_kv, N, d,
                                int(bool(causal)), float(scale), int(mode), _stream(stream)), "attn_bwd_varlen")
+
+
+def attn_packed_workspace_bytes(B, H, H_kv, N_max, d, backward):
+    return int(lib.attn_packed_workspace_bytes(B, H, H_kv, N_max, d, int(bool(backward))))
+
+
+def attn_fwd_packed(q, k, v, o, lse, cu_seqlens, workspace, workspace_bytes, B, H, H_kv, T, N_max, d, causal, scale,
+                    mode=0, stream=None):
+    _check(lib.attn_fwd_packed(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(cu_seqlens), _ptr(workspace),
+                               int(workspace_bytes), B, H, H_kv, T, N_max, d, int(bool(causal)), float(scale), int(mode),
+                               _stream(stream)), "attn_fwd_packed")
+
+
+def attn_bwd_packed(q, k, v, o, dO, lse, dq, dk, dv, delta, cu_seqlens, workspace, workspace_bytes, B, H, H_kv, T, N_max,
+                    d, causal, scale, mode=0, stream=None):
+    _check(lib.attn_bwd_packed(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(dO), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv),
+                               _ptr(delta), _ptr(cu_seqlens), _ptr(workspace), int(workspace_bytes), B, H, H_kv, T, N_max,
+                               d, int(bool(causal)), float(scale), int(mode), _stream(stream)), "attn_bwd_packed")
 
 
 def attn_bwd_workspace_bytes(B, H, N, d):

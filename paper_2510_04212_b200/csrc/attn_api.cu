@@ -11,6 +11,7 @@
 #include "../../include/attn.h"
 #include "bwd_kernel.cuh"
 #include "bwd_kernel_d64.cuh"
+#include "packed_copy_kernel.cuh"
 #include "bwd_kernel_d128.cuh"
 #include "delta_dp_kernel.cuh"
 #include "fwd_kernel.cuh"
@@ -541,6 +542,141 @@ int attn_bwd_varlen(const void* q, const void* k, const void* v, const void* o, 
     if (!seqlens) return ATTN_ERR_NULL;
     return bwd_stage_impl(ATTN_BWD_STAGE_ALL, q, k, v, o, dO, lse, dq, dk, dv, delta, workspace, workspace_bytes,
                           B, H, H_kv, N, N, seqlens, d, causal, scale, mode, stream);
+}
+
+// ---------------------------------------------------------------- packed variable-length batches
+// The packed entry points copy between the caller's packed tensors and padded tensors in the workspace and run the
+// per-batch-length kernels on those.  Layout of the workspace (every part a multiple of 256 bytes):
+//   seqlens int[B] | q | k | v | o | lse            (forward)
+//   ... | dO | dq | dk | dv | delta | FP32 dQ accumulator of attn_bwd_workspace_bytes(B, H, N_max, d)   (backward)
+extern "C++" {
+namespace {
+struct PackedLayout {
+    size_t seqlens, q, k, v, o, lse, dO, dq, dk, dv, delta, acc, total_fwd, total_bwd;
+};
+size_t round256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+PackedLayout packed_layout(int B, int H, int Hkv, int N, int d)
+{
+    PackedLayout L;
+    const size_t eq = round256(static_cast<size_t>(B) * H * N * d * 2), ekv = round256(static_cast<size_t>(B) * Hkv * N * d * 2);
+    const size_t vec = round256(static_cast<size_t>(B) * H * N * 4);
+    size_t p = 0;
+    L.seqlens = p; p += round256(static_cast<size_t>(B) * 4);
+    L.q = p; p += eq;
+    L.k = p; p += ekv;
+    L.v = p; p += ekv;
+    L.o = p; p += eq;
+    L.lse = p; p += vec;
+    L.total_fwd = p;
+    L.dO = p; p += eq;
+    L.dq = p; p += eq;
+    L.dk = p; p += ekv;
+    L.dv = p; p += ekv;
+    L.delta = p; p += vec;
+    L.acc = p; p += round256(attn_bwd_workspace_bytes(B, H, N, d));
+    L.total_bwd = p;
+    return L;
+}
+int check_packed(const int* cu, void* workspace, int B, int H, int Hkv, int T, int N, int d)
+{
+    if (!cu) return ATTN_ERR_NULL;
+    if (int e = check_shape(B, H, N, d)) return e;
+    if (Hkv < 1 || H % Hkv != 0 || T < 1) return ATTN_ERR_SHAPE;
+    if (static_cast<long long>(T) * H >= (1ll << 31)) return ATTN_ERR_SHAPE;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return ATTN_ERR_WORKSPACE;
+    return ATTN_OK;
+}
+template <bool TO_PADDED>
+int copy_rows(void* padded, const void* packed, const int* cu, int B, int Hx, int N, int d, cudaStream_t st)
+{
+    const int cpr = d / 8;
+    const long long n = static_cast<long long>(B) * Hx * N * cpr;
+    attn::packed_rows_kernel<TO_PADDED><<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+        static_cast<uint4*>(padded), static_cast<uint4*>(const_cast<void*>(packed)), cu, Hx, N, cpr, n);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+template <bool TO_PADDED>
+int copy_vec(float* padded, const float* packed, const int* cu, int B, int H, int N, int T, cudaStream_t st)
+{
+    const long long n = static_cast<long long>(B) * H * N;
+    attn::packed_vec_kernel<TO_PADDED><<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+        padded, const_cast<float*>(packed), cu, H, N, T, n);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+}  // namespace
+}  // extern "C++"
+
+size_t attn_packed_workspace_bytes(int B, int H, int H_kv, int N_max, int d, int backward)
+{
+    if (check_shape(B, H, N_max, d) != ATTN_OK || H_kv < 1 || H % H_kv != 0) return 0;
+    const PackedLayout L = packed_layout(B, H, H_kv, N_max, d);
+    return backward ? L.total_bwd : L.total_fwd;
+}
+
+int attn_fwd_packed(const void* q, const void* k, const void* v, void* o, float* lse, const int* cu_seqlens,
+                    void* workspace, size_t workspace_bytes, int B, int H, int H_kv, int T, int N_max, int d,
+                    int causal, float scale, int mode, void* stream)
+{
+    if (!q || !k || !v || !o || !lse) return ATTN_ERR_NULL;
+    if (int e = check_packed(cu_seqlens, workspace, B, H, H_kv, T, N_max, d)) return e;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return ATTN_ERR_ALIGN;
+    const PackedLayout L = packed_layout(B, H, H_kv, N_max, d);
+    if (workspace_bytes < L.total_fwd) return ATTN_ERR_WORKSPACE;
+    if (int e = check_device()) return e;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* seqlens = reinterpret_cast<int*>(w + L.seqlens);
+    attn::packed_seqlens_kernel<<<(B + 127) / 128, 128, 0, st>>>(cu_seqlens, seqlens, B, N_max);
+    if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_CUDA;
+    if (int e = copy_rows<true>(w + L.q, q, cu_seqlens, B, H, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.k, k, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.v, v, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (int e = fwd_impl(w + L.q, w + L.k, w + L.v, w + L.o, reinterpret_cast<float*>(w + L.lse), nullptr, B, H, H_kv,
+                         N_max, N_max, seqlens, d, causal, scale, mode, stream))
+        return e;
+    if (int e = copy_rows<false>(w + L.o, o, cu_seqlens, B, H, N_max, d, st)) return e;
+    return copy_vec<false>(reinterpret_cast<float*>(w + L.lse), lse, cu_seqlens, B, H, N_max, T, st);
+}
+
+int attn_bwd_packed(const void* q, const void* k, const void* v, const void* o, const void* dO, const float* lse,
+                    void* dq, void* dk, void* dv, float* delta, const int* cu_seqlens,
+                    void* workspace, size_t workspace_bytes, int B, int H, int H_kv, int T, int N_max, int d,
+                    int causal, float scale, int mode, void* stream)
+{
+    if (!q || !k || !v || !o || !dO || !lse || !dq || !dk || !dv || !delta) return ATTN_ERR_NULL;
+    if (int e = check_packed(cu_seqlens, workspace, B, H, H_kv, T, N_max, d)) return e;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dO) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return ATTN_ERR_ALIGN;
+    const PackedLayout L = packed_layout(B, H, H_kv, N_max, d);
+    if (workspace_bytes < L.total_bwd) return ATTN_ERR_WORKSPACE;
+    if (int e = check_device()) return e;
+    uint8_t* w = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* seqlens = reinterpret_cast<int*>(w + L.seqlens);
+    float* lse_p = reinterpret_cast<float*>(w + L.lse);
+    float* delta_p = reinterpret_cast<float*>(w + L.delta);
+    const bool given = (mode & ATTN_MODE_FLAG_DELTA_GIVEN) != 0;
+    attn::packed_seqlens_kernel<<<(B + 127) / 128, 128, 0, st>>>(cu_seqlens, seqlens, B, N_max);
+    if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_CUDA;
+    if (int e = copy_rows<true>(w + L.q, q, cu_seqlens, B, H, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.k, k, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.v, v, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.o, o, cu_seqlens, B, H, N_max, d, st)) return e;
+    if (int e = copy_rows<true>(w + L.dO, dO, cu_seqlens, B, H, N_max, d, st)) return e;
+    if (int e = copy_vec<true>(lse_p, lse, cu_seqlens, B, H, N_max, T, st)) return e;
+    if (given)
+        if (int e = copy_vec<true>(delta_p, delta, cu_seqlens, B, H, N_max, T, st)) return e;
+    if (int e = bwd_stage_impl(ATTN_BWD_STAGE_ALL, w + L.q, w + L.k, w + L.v, w + L.o, w + L.dO, lse_p, w + L.dq, w + L.dk,
+                               w + L.dv, delta_p, w + L.acc, L.total_bwd - L.acc, B, H, H_kv, N_max, N_max, seqlens, d,
+                               causal, scale, mode, stream))
+        return e;
+    if (int e = copy_rows<false>(w + L.dq, dq, cu_seqlens, B, H, N_max, d, st)) return e;
+    if (int e = copy_rows<false>(w + L.dk, dk, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (int e = copy_rows<false>(w + L.dv, dv, cu_seqlens, B, H_kv, N_max, d, st)) return e;
+    if (!given)
+        if (int e = copy_vec<false>(delta_p, delta, cu_seqlens, B, H, N_max, T, st)) return e;
+    return ATTN_OK;
 }
 
 int attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* dO, const float* lse,

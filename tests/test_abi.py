@@ -92,6 +92,10 @@ def test_argument_validation_comes_before_any_device_work():
     assert lib.attn_fwd_o_f32(p, p, p, p, p, p, 1, 1, 100, 64, 1, 0.125, 0, None) == -2
     assert lib.attn_bwd_delta_f32(None, p, p, 1, 1, 128, 64, None) == -1
     assert lib.attn_bwd_delta_f32(p, p, p, 1, 1, 128, 96, None) == -2
+    assert lib.attn_fwd_packed(p, p, p, p, p, None, p, 1 << 30, 2, 4, 2, 300, 256, 64, 1, 0.125, 0, None) == -1
+    assert lib.attn_fwd_packed(p, p, p, p, p, p, p, 16, 2, 4, 2, 300, 256, 64, 1, 0.125, 0, None) == -5
+    assert lib.attn_bwd_packed(p, p, p, p, p, p, p, p, p, None, p, p, 1 << 30, 2, 4, 2, 300, 256, 64, 1, 0.125, 0, None) == -1
+    assert lib.attn_bwd_packed(p, p, p, p, p, p, p, p, p, p, p, p, 1 << 20, 2, 4, 2, 300, 200, 64, 1, 0.125, 0, None) == -2
     assert lib.attn_bwd_preprocess(None, p, p, 1, 1, 128, 64, None) == -1
     assert lib.attn_bwd_preprocess(p, p, p, 1, 1, 128, 32, None) == -2
 
