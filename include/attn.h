@@ -168,6 +168,24 @@ int attn_fwd_pbar_format(const void* q, const void* k, const void* v, void* o, f
                          void* stream);
 
 /*
+ * The P-bar V product of the forward pass on the 8-bit tensor path: the setting the paper names as future work
+ * (Sec. 5: FP8 training), built so that its numerics and its speed can be measured; not part of the paper's method.
+ *
+ * attn_quantize_v_e4m3:  v_t[b][h][c][n] = e4m3(v[b][h][n][c] * v_scale)   (round to nearest even, saturating at 448)
+ *   in : v         BF16 [B][H][N][d];   v_scale > 0 (ATTN_ERR_PARAM otherwise)
+ *   out: v_t_e4m3  E4M3 [B][H][d][N]    one byte per element, transposed, 16-byte aligned
+ * attn_fwd_fp8pv:  attn_fwd with P-bar = e4m3(exp(S - m)) (instead of BF16) and V taken from v_t_e4m3; the product
+ *   O-bar += P-bar V runs as tcgen05.mma kind::f8f6f4 with FP32 accumulation (the products of two E4M3 values are
+ *   exact in FP32).  S = Q K^T stays BF16 x BF16, all statistics stay FP32, l sums the rounded P-bar, and
+ *   O = bf16(bf16(v_descale * O-bar) / l): pass v_descale = 1 / v_scale.  mode: 0 or ATTN_MODE_STABILISED only
+ *   (other bits: ATTN_ERR_MODE).  The result equals attn_fwd_pbar_format(..., ATTN_PBAR_E4M3) run on the
+ *   dequantised V, up to the order of the FP32 sums.  Other arguments, checks and errors as attn_fwd.
+ */
+int attn_quantize_v_e4m3(const void* v, void* v_t_e4m3, int B, int H, int N, int d, float v_scale, void* stream);
+int attn_fwd_fp8pv(const void* q, const void* k, const void* v_t_e4m3, void* o, float* lse,
+                   int B, int H, int N, int d, int causal, float scale, int mode, float v_descale, void* stream);
+
+/*
  * delta = rowsum(dO o O), the preprocessing step of Algorithm 2 (Sec. 2.2).
  *   in : o, dO   BF16 [B][H][N][d]
  *   out: delta   FP32 [B][H][N]

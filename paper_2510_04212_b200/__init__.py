@@ -13,12 +13,12 @@ import os
 
 from . import build as _build
 
-__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
+__all__ = ["AttnError", "attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_quantize_v_e4m3", "attn_fwd_fp8pv", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes",
            "attn_get_tiles", "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout",
            "attn_strerror", "lib", "LIB_PATH", "EXPORTS"]
 
 LIB_PATH = _build.LIB
-EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
+EXPORTS = ("attn_fwd", "attn_fwd_count_ones", "attn_fwd_o_f32", "attn_bwd_delta_f32", "attn_quantize_v_e4m3", "attn_fwd_fp8pv", "attn_fwd_pbar_format", "attn_bwd", "attn_bwd_stage", "attn_bwd_static", "attn_fwd_gqa", "attn_bwd_gqa", "attn_fwd_padded", "attn_bwd_padded", "attn_fwd_varlen", "attn_bwd_varlen", "attn_fwd_packed", "attn_bwd_packed", "attn_packed_workspace_bytes", "attn_bwd_preprocess", "attn_bwd_delta_dp", "attn_bwd_workspace_bytes", "attn_get_tiles",
            "attn_set_mitigation", "attn_get_mitigation", "attn_set_guard_max_shift", "attn_get_guard_max_shift", "attn_last_device_status", "attn_selftest_wait_timeout", "attn_strerror")
 
 
@@ -54,6 +54,10 @@ def _load():
     L.attn_fwd_packed.argtypes = [vp, vp, vp, vp, fp, vp, vp, sz, i, i, i, i, i, i, i, f, i, vp]
     L.attn_bwd_packed.restype = i
     L.attn_bwd_packed.argtypes = [vp, vp, vp, vp, vp, fp, vp, vp, vp, fp, vp, vp, sz, i, i, i, i, i, i, i, f, i, vp]
+    L.attn_quantize_v_e4m3.restype = i
+    L.attn_quantize_v_e4m3.argtypes = [vp, vp, i, i, i, i, f, vp]
+    L.attn_fwd_fp8pv.restype = i
+    L.attn_fwd_fp8pv.argtypes = [vp, vp, vp, vp, fp, i, i, i, i, i, f, i, f, vp]
     L.attn_bwd_preprocess.restype = i
     L.attn_bwd_preprocess.argtypes = [vp, vp, fp, i, i, i, i, vp]
     L.attn_bwd.restype = i
@@ -153,6 +157,16 @@ def attn_fwd_o_f32(q, k, v, o, lse, o_f32, B, H, N, d, causal, scale, mode, stre
 def attn_bwd_delta_f32(o_f32, dO, delta, B, H, N, d, stream=None):
     _check(lib.attn_bwd_delta_f32(_ptr(o_f32), _ptr(dO), _ptr(delta), B, H, N, d, _stream(stream)),
            "attn_bwd_delta_f32")
+
+
+def attn_quantize_v_e4m3(v, v_t_e4m3, B, H, N, d, v_scale=1.0, stream=None):
+    _check(lib.attn_quantize_v_e4m3(_ptr(v), _ptr(v_t_e4m3), B, H, N, d, float(v_scale), _stream(stream)),
+           "attn_quantize_v_e4m3")
+
+
+def attn_fwd_fp8pv(q, k, v_t_e4m3, o, lse, B, H, N, d, causal, scale, mode=0, v_descale=1.0, stream=None):
+    _check(lib.attn_fwd_fp8pv(_ptr(q), _ptr(k), _ptr(v_t_e4m3), _ptr(o), _ptr(lse), B, H, N, d, int(bool(causal)),
+                              float(scale), int(mode), float(v_descale), _stream(stream)), "attn_fwd_fp8pv")
 
 
 def attn_bwd_preprocess(o, dO, delta, B, H, N, d, stream=None):

@@ -6,7 +6,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libattn_b200.so")
 SOURCES = [os.path.join(CSRC, "attn_api.cu")]
-HEADERS = [os.path.join(CSRC, n) for n in ("ptx.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "bwd_kernel_d64.cuh", "bwd_kernel_d128.cuh", "delta_dp_kernel.cuh", "selftest_kernel.cuh", "packed_copy_kernel.cuh")] + [
+HEADERS = [os.path.join(CSRC, n) for n in ("ptx.cuh", "fwd_kernel.cuh", "bwd_kernel.cuh", "bwd_kernel_d64.cuh", "bwd_kernel_d128.cuh", "delta_dp_kernel.cuh", "selftest_kernel.cuh", "packed_copy_kernel.cuh", "quantize_v_kernel.cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "attn.h")]
 
 

@@ -12,6 +12,7 @@
 #include "bwd_kernel.cuh"
 #include "bwd_kernel_d64.cuh"
 #include "packed_copy_kernel.cuh"
+#include "quantize_v_kernel.cuh"
 #include "bwd_kernel_d128.cuh"
 #include "delta_dp_kernel.cuh"
 #include "fwd_kernel.cuh"
@@ -66,6 +67,20 @@ bool make_map(CUtensorMap* m, const void* base, long long rows, int d, int box_r
     const cuuint32_t estr[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// V transposed, one-byte elements: [rows = B*H*d][N keys]; one box = d rows x 64 keys (64 bytes), 64-byte swizzle.
+bool make_map_vt_u8(CUtensorMap* m, const void* base, long long rows, int N, int d)
+{
+    EncodeTiledFn enc = get_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(N)};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(d)};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -162,12 +177,12 @@ cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t sme
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
-template <int D, int MODE, bool CAUSAL, bool COUNT, bool PADDED = false>
+template <int D, int MODE, bool CAUSAL, bool COUNT, bool PADDED = false, bool FP8PV = false>
 int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
                const attn::FwdParams& prm, cudaStream_t st)
 {
     using Cfg = attn::FwdCfg<D>;
-    constexpr auto kern = attn::attn_fwd_kernel<D, MODE, CAUSAL, COUNT, PADDED>;
+    constexpr auto kern = attn::attn_fwd_kernel<D, MODE, CAUSAL, COUNT, PADDED, FP8PV>;
     if (int e = ensure_dynamic_smem<kern>(Cfg::SMEM_BYTES)) return e;
     return launch_pdl(kern, dim3(prm.Tr * prm.BH), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tq, tk, tv, to, prm) == cudaSuccess
                ? ATTN_OK : ATTN_ERR_CUDA;
@@ -243,8 +258,9 @@ extern "C" {
 // attn_fwd and attn_fwd_count_ones: `ones` == nullptr selects the instantiations without the counter
 static int fwd_impl(const void* q, const void* k, const void* v, void* o, float* lse, int* ones,
                     int B, int H, int Hkv, int N, int seqlen, const int* seqlens, int d, int causal, float scale, int mode,
-                    void* stream, int pbar_fmt = ATTN_PBAR_BF16, float* o_f32 = nullptr)
+                    void* stream, int pbar_fmt = ATTN_PBAR_BF16, float* o_f32 = nullptr, float fp8_v_descale = 0.0f)
 {
+    const bool fp8pv = fp8_v_descale != 0.0f;       // v is then V^T in E4M3, [B][H][d][N]
     if (pbar_fmt != ATTN_PBAR_BF16 && pbar_fmt != ATTN_PBAR_E4M3 && pbar_fmt != ATTN_PBAR_E5M2) return ATTN_ERR_MODE;
     if (!q || !k || !v || !o || !lse) return ATTN_ERR_NULL;
     if (int e = check_shape(B, H, N, d)) return e;
@@ -262,8 +278,9 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     CUtensorMap tq, tk, tv, to;
     const int bc = attn::FwdCfg<64>::BC;
     const long long kvrows = static_cast<long long>(B) * Hkv * N;
-    if (!make_map(&tq, q, rows, d, 128) || !make_map(&tk, k, kvrows, d, bc) || !make_map(&tv, v, kvrows, d, bc) ||
-        !make_map(&to, o, rows, d, 128))
+    if (!make_map(&tq, q, rows, d, 128) || !make_map(&tk, k, kvrows, d, bc) || !make_map(&to, o, rows, d, 128))
+        return ATTN_ERR_CUDA;
+    if (!(fp8pv ? make_map_vt_u8(&tv, v, static_cast<long long>(B) * Hkv * d, N, d) : make_map(&tv, v, kvrows, d, bc)))
         return ATTN_ERR_CUDA;
 
     attn::FwdParams prm;
@@ -283,8 +300,22 @@ static int fwd_impl(const void* q, const void* k, const void* v, void* o, float*
     prm.beta = g_beta.load();
     prm.eps = g_eps.load();
     prm.guard_cap = (mode & ATTN_MODE_FLAG_GUARDED) ? g_guard_cap.load() : 0.0f;
+    prm.v_descale = fp8_v_descale;
     prm.status = status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (fp8pv) {
+        const bool m1 = (mode & ATTN_MODE_STABILISED) != 0;
+        if (d == 64) {
+            if (causal) return m1 ? launch_fwd<64, 1, true, false, false, true>(tq, tk, tv, to, prm, st)
+                                  : launch_fwd<64, 0, true, false, false, true>(tq, tk, tv, to, prm, st);
+            return m1 ? launch_fwd<64, 1, false, false, false, true>(tq, tk, tv, to, prm, st)
+                      : launch_fwd<64, 0, false, false, false, true>(tq, tk, tv, to, prm, st);
+        }
+        if (causal) return m1 ? launch_fwd<128, 1, true, false, false, true>(tq, tk, tv, to, prm, st)
+                              : launch_fwd<128, 0, true, false, false, true>(tq, tk, tv, to, prm, st);
+        return m1 ? launch_fwd<128, 1, false, false, false, true>(tq, tk, tv, to, prm, st)
+                  : launch_fwd<128, 0, false, false, false, true>(tq, tk, tv, to, prm, st);
+    }
     const int key = (d == 128 ? 8 : 0) | ((mode & ATTN_MODE_STABILISED) ? 4 : 0) | (causal ? 2 : 0) | ((ones || o_f32) ? 1 : 0);
     // full attention over a sequence that ends inside a 64-key tile: the instantiations that mask the rest of that tile
     if (!causal && (seqlen % bc != 0 || seqlens)) {
@@ -328,6 +359,31 @@ int attn_fwd_pbar_format(const void* q, const void* k, const void* v, void* o, f
 {
     if (!ones) return ATTN_ERR_NULL;
     return fwd_impl(q, k, v, o, lse, ones, B, H, H, N, N, nullptr, d, causal, scale, mode, stream, pbar_format);
+}
+
+int attn_quantize_v_e4m3(const void* v, void* v_t_e4m3, int B, int H, int N, int d, float v_scale, void* stream)
+{
+    if (!v || !v_t_e4m3) return ATTN_ERR_NULL;
+    if (int e = check_shape(B, H, N, d)) return e;
+    if (!(v_scale > 0.0f) || !isfinite(v_scale)) return ATTN_ERR_PARAM;
+    if (!aligned16(v) || !aligned16(v_t_e4m3)) return ATTN_ERR_ALIGN;
+    if (int e = check_device()) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(static_cast<unsigned>(N / (16 * (256 / d))), static_cast<unsigned>(B * H));
+    if (d == 64)
+        attn::quantize_v_e4m3_kernel<64><<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(v), static_cast<uint8_t*>(v_t_e4m3), N, v_scale);
+    else
+        attn::quantize_v_e4m3_kernel<128><<<grid, 256, 0, st>>>(static_cast<const uint16_t*>(v), static_cast<uint8_t*>(v_t_e4m3), N, v_scale);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
+}
+
+int attn_fwd_fp8pv(const void* q, const void* k, const void* v_t_e4m3, void* o, float* lse,
+                   int B, int H, int N, int d, int causal, float scale, int mode, float v_descale, void* stream)
+{
+    if (!(v_descale > 0.0f) || !isfinite(v_descale)) return ATTN_ERR_PARAM;
+    if (mode & ~ATTN_MODE_STABILISED) return ATTN_ERR_MODE;
+    return fwd_impl(q, k, v_t_e4m3, o, lse, nullptr, B, H, H, N, N, nullptr, d, causal, scale, mode, stream, ATTN_PBAR_BF16,
+                    nullptr, v_descale);
 }
 
 int attn_fwd_o_f32(const void* q, const void* k, const void* v, void* o, float* lse, float* o_f32,

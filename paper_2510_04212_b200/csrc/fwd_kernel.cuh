@@ -76,13 +76,17 @@ struct FwdParams {
     int group;                 // query heads per key/value head (grouped-query attention; 1 = multi-head)
     float scale, beta, eps;
     float guard_cap;           // > 0: guarded variant of the tie rule (mode 1 only)
+    float v_descale;           // FP8PV instantiations only: O-bar is multiplied by this before it is rounded
     int* status;
 };
 
 // COUNT (compile time): also count, per row, the entries of P-bar that are exactly 1 (Sec. 3.3.2)
 // PADDED (compile time; full attention only, the causal mask already hides the padding keys from every sequence row):
 // the sequence may end inside a key tile, whose remaining keys are masked
-template <int D, int MODE, bool CAUSAL, bool COUNT = false, bool PADDED = false>
+// FP8PV (compile time): P-bar is rounded to E4M3 and multiplied with an E4M3 V on the 8-bit tensor path
+// (tcgen05.mma kind::f8f6f4).  tmV then describes V transposed, [B*H*d rows][N keys] of one-byte elements, so that a
+// key tile is a K-major operand ([d rows][64 keys], 64-byte rows, 64-byte swizzle).
+template <int D, int MODE, bool CAUSAL, bool COUNT = false, bool PADDED = false, bool FP8PV = false>
 __global__ void __launch_bounds__(FwdCfg<D>::THREADS, FwdCfg<D>::CTAS_PER_SM)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -160,9 +164,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int p = 0; p < Cfg::PANELS; ++p)
                     tma_load_2d(sK0 + s * Cfg::KV_BYTES + p * Cfg::KV_PANEL_BYTES, &tmK, bar(K_FULL + s), p * 64, kvrow0 + j * Cfg::BC);
                 if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1, &abort_flag)) break;
-                mbar_expect_tx(bar(V_FULL + s), Cfg::KV_BYTES);
-                for (int p = 0; p < Cfg::PANELS; ++p)
-                    tma_load_2d(sV0 + s * Cfg::KV_BYTES + p * Cfg::KV_PANEL_BYTES, &tmV, bar(V_FULL + s), p * 64, kvrow0 + j * Cfg::BC);
+                if constexpr (FP8PV) {                      // one box: 64 keys (bytes) x d rows of the transposed V
+                    mbar_expect_tx(bar(V_FULL + s), D * Cfg::BC);
+                    tma_load_2d(sV0 + s * Cfg::KV_BYTES, &tmV, bar(V_FULL + s), j * Cfg::BC, (bh / prm.group) * D);
+                } else {
+                    mbar_expect_tx(bar(V_FULL + s), Cfg::KV_BYTES);
+                    for (int p = 0; p < Cfg::PANELS; ++p)
+                        tma_load_2d(sV0 + s * Cfg::KV_BYTES + p * Cfg::KV_PANEL_BYTES, &tmV, bar(V_FULL + s), p * 64, kvrow0 + j * Cfg::BC);
+                }
             }
         }
         __syncwarp();
@@ -175,7 +184,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             // 16-byte units) moves, by compile-time constants per k-step plus the stage
             const uint64_t dQ0 = make_smem_desc(sQ, 16, 1024);
             const uint64_t dK0 = make_smem_desc(sK0, 16, 1024);
-            const uint64_t dV0 = make_smem_desc(sV0, Cfg::KV_PANEL_BYTES, 1024);
+            const uint64_t dV0 = FP8PV ? make_smem_desc_sw64(sV0, 16, 512) : make_smem_desc(sV0, Cfg::KV_PANEL_BYTES, 1024);
+            constexpr uint32_t idesc_PV8 = make_idesc_e4m3(128, D);
             auto issue_S = [&](int j) -> bool {           // S(j) = Q K_j^T
                 const int s = j % Cfg::STAGES, ph = (j / Cfg::STAGES) & 1;
                 if (!mbar_wait(bar(K_FULL + s), ph, &abort_flag)) return false;
@@ -203,10 +213,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 const uint64_t dV = dV0 + static_cast<uint64_t>((s * Cfg::KV_BYTES) >> 4);
                 const uint32_t tP = tmem_S + sb * 64;
                 // O-bar += P-bar(j) V_j: V_j as the B operand, N = d contiguous (MN-major), 16 key rows per step
-                mma_ts(tmem_O, tP, dV, idesc_PV, (j > 0) ? 1u : 0u);
+                if constexpr (FP8PV) {
+                    // 8-bit operands: 32 keys per step (8 TMEM columns of P-bar, 32 bytes along a row of V^T)
+                    mma_ts_f8(tmem_O, tP, dV, idesc_PV8, (j > 0) ? 1u : 0u);
+                    mma_ts_f8(tmem_O, tP + 8, dV + (32 >> 4), idesc_PV8, 1u);
+                } else {
+                    mma_ts(tmem_O, tP, dV, idesc_PV, (j > 0) ? 1u : 0u);
 #pragma unroll
-                for (int k = 1; k < Cfg::BC / 16; ++k)
-                    mma_ts(tmem_O, tP + k * 8, dV + ((k * 2048) >> 4), idesc_PV, 1u);
+                    for (int k = 1; k < Cfg::BC / 16; ++k)
+                        mma_ts(tmem_O, tP + k * 8, dV + ((k * 2048) >> 4), idesc_PV, 1u);
+                }
                 mma_commit(pv_done_bar(j));
                 mma_commit(bar(V_EMPTY + s));
                 // the next S for this buffer overwrites it; the MMAs just issued consume its P-bar(j) first
@@ -351,6 +367,26 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int h = 0; h < 2; ++h) {
                     tmem_ld32(tS + h * 32, r);
                     tmem_wait_ld();
+                    if constexpr (FP8PV) {
+                        uint32_t pk8[8];
+    #pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            float x0, x1, x2, x3;
+                            exp_arg(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+                            exp_arg(x2, x3, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+                            float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                            if (DIAG) {
+                                if (h * 32 + c > vis) p0 = 0.0f;
+                                if (h * 32 + c + 1 > vis) p1 = 0.0f;
+                                if (h * 32 + c + 2 > vis) p2 = 0.0f;
+                                if (h * 32 + c + 3 > vis) p3 = 0.0f;
+                            }
+                            pk8[c >> 2] = pack_e4m3x4(p0, p1, p2, p3);
+                            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                        }
+                        // E4M3 P-bar columns [8h, 8h + 8) overlay score columns read in this or the earlier step
+                        tmem_st8(tS + h * 8, pk8);
+                    } else {
                     uint32_t pk[16];
     #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
@@ -371,6 +407,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     // P-bar columns [16h, 16h+16) overlay score columns [16h, 16h+16): for h = 0 those are in registers
                     // already; for h = 1 they are columns [16,32), read in the h = 0 step -- nothing still needed is lost
                     tmem_st16(tS + h * 16, pk);
+                    }
                 }
                 l = a * l + ((sum0 + sum1) + (sum2 + sum3));
             } else {
@@ -454,6 +491,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 // ---- P-bar = bf16(exp(S - m)) -> TMEM (over S); l += FP32 sum of the rounded values
                 float sum0 = 0.0f, sum1 = 0.0f, sum2 = 0.0f, sum3 = 0.0f;
                 auto exp_chunk = [&](const uint32_t (&r)[32], int h) {
+                    if constexpr (FP8PV) {
+                        uint32_t pk8[8];
+    #pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            float x0, x1, x2, x3;
+                            exp_arg(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]));
+                            exp_arg(x2, x3, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+                            float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                            if (DIAG) {
+                                if (h * 32 + c > vis) p0 = 0.0f;
+                                if (h * 32 + c + 1 > vis) p1 = 0.0f;
+                                if (h * 32 + c + 2 > vis) p2 = 0.0f;
+                                if (h * 32 + c + 3 > vis) p3 = 0.0f;
+                            }
+                            pk8[c >> 2] = pack_e4m3x4(p0, p1, p2, p3);
+                            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                        }
+                        tmem_st8(tS + h * 8, pk8);
+                    } else {
                     uint32_t pk[16];
     #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
@@ -472,6 +528,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                         else              add_bf16x2_halves(sum2, sum3, w);
                     }
                     tmem_st16(tS + h * 16, pk);
+                    }
                 };
                 exp_chunk(ra, 0);
                 exp_chunk(rb, 1);
@@ -552,6 +609,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
                     float o0 = __uint_as_float(r[c]), o1 = __uint_as_float(r[c + 1]);
+                    if constexpr (FP8PV) { o0 *= prm.v_descale; o1 *= prm.v_descale; }
                     if (!prm.single_rounding) {                   // O-bar -> BF16 (the paper's rounding point)
                         const uint32_t ob = pack_bf16(o0, o1);
                         o0 = bf16_lo(ob);

@@ -177,6 +177,25 @@ __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
 }
 
 // Round two FP32 values to nearest-even in an 8-bit format (E4M3: fmt == 1, otherwise E5M2) and return them as FP32.
+// Four FP32 values -> E4M3 (nearest even, saturating), packed with p0 in the lowest byte; the arguments are
+// replaced by the rounded values.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float& p0, float& p1, float& p2, float& p3) {
+    uint32_t w;
+    asm("{ .reg .b16 h0, h1, a, b; .reg .b32 w0, w1;\n"
+        "cvt.rn.satfinite.e4m3x2.f32 h0, %6, %5;\n"
+        "cvt.rn.satfinite.e4m3x2.f32 h1, %8, %7;\n"
+        "mov.b32 %0, {h0, h1};\n"
+        "cvt.rn.f16x2.e4m3x2 w0, h0;\n"
+        "cvt.rn.f16x2.e4m3x2 w1, h1;\n"
+        "mov.b32 {a, b}, w0;\n"
+        "cvt.f32.f16 %1, a;\n"
+        "cvt.f32.f16 %2, b;\n"
+        "mov.b32 {a, b}, w1;\n"
+        "cvt.f32.f16 %3, a;\n"
+        "cvt.f32.f16 %4, b; }"
+        : "=r"(w), "=f"(p0), "=f"(p1), "=f"(p2), "=f"(p3) : "f"(p0), "f"(p1), "f"(p2), "f"(p3));
+    return w;
+}
 __device__ __forceinline__ void round_fp8x2(float& a, float& b, int fmt) {
     if (fmt == 1)
         asm("{ .reg .b16 h, lo, hi; .reg .b32 w;\n"
@@ -248,6 +267,12 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -275,6 +300,21 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     d |= static_cast<uint64_t>(2) << 61;
     return d;
 }
+// The same for a K-major operand whose rows are 64 bytes (64 one-byte elements) in the 64-byte swizzle
+// (layout type 4; 8-row groups are sbo_bytes = 512 apart).
+__device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(4) << 61;
+    return d;
+}
+// Instruction descriptor for kind::f8f6f4 with E4M3 A and B (format code 0), both K-major, FP32 accumulate.
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N) {
+    return (1u << 4) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
+}
 // Instruction descriptor for kind::f16 with BF16 A/B and FP32 accumulate.
 //   [4,6) D format 1=F32; [7,10) A format 1=BF16; [10,13) B format 1=BF16;
 //   [15] A major (0=K,1=MN); [16] B major; [17,23) N>>3; [24,29) M>>4.
@@ -296,6 +336,14 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem], 8-bit operands (32 per step along K; A: four per 32-bit TMEM column)
+__device__ __forceinline__ void mma_ts_f8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // Arrive on an mbarrier when every MMA issued so far by this thread has completed.
