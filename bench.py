@@ -275,6 +275,18 @@ def context_libs(torch, steps=20):
                 torch.cuda.synchronize()
                 ms = e0.elapsed_time(e1) / steps
                 out[label] = {"ms_per_step": ms, "tflops": (f_fwd + f_bwd) / (ms * 1e-3) / 1e12, "how": how}
+                # the forward alone (eager calls back to back: no autograd graph to build, the launches queue ahead)
+                with torch.no_grad():
+                    fwd_only = lambda i: F.scaled_dot_product_attention(*sets[i % len(sets)][:3], is_causal=causal)
+                    for i in range(3):
+                        fwd_only(i)
+                    torch.cuda.synchronize()
+                    e0.record()
+                    for i in range(steps):
+                        fwd_only(i)
+                    e1.record()
+                    torch.cuda.synchronize()
+                out[label]["fwd_ms"] = e0.elapsed_time(e1) / steps
         except Exception as e:            # a back end that is not available for this shape on this machine
             out[label] = {"unavailable": str(e).splitlines()[0][:200]}
     return out
