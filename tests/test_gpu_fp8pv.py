@@ -17,38 +17,7 @@ def _env():
     return _gpu_util, attn
 
 
-def e4m3_table():
-    """The 256 values of the E4M3 format by its definition (bias 7, subnormals, no infinity, S.1111.111 = NaN)."""
-    t = np.empty(256, np.float64)
-    for b in range(256):
-        s, e, m = b >> 7, (b >> 3) & 15, b & 7
-        v = (m / 8.0) * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
-        t[b] = np.nan if (e == 15 and m == 7) else (-v if s else v)
-    return t
-
-
-def quantize_e4m3(x):
-    """Nearest E4M3 value of |x| (ties to the even code, saturating at 448) with the sign of x: brute force over the
-    table of the non-negative codes."""
-    tab = e4m3_table()
-    codes = np.arange(0x7F)                                            # 0 .. 0x7E: the finite non-negative values
-    vals = tab[codes]
-    x = np.asarray(x, np.float64)
-    mag = np.minimum(np.abs(x), 448.0)
-    dist = np.abs(mag[..., None] - vals)
-    best = dist.min(-1, keepdims=True)
-    cand = np.where(dist == best, codes, 1 << 20)                      # all nearest codes (two on a tie)
-    even = np.where((cand & 1) == 0, cand, 1 << 20)
-    pick = np.where(even.min(-1) < (1 << 20), even.min(-1), cand.min(-1))
-    return (pick | np.where(np.signbit(x), 0x80, 0)).astype(np.uint8)
-
-
-def test_host_quantiser_agrees_with_the_oracle_routine():
-    rng = np.random.default_rng(5)
-    xs = np.concatenate([rng.normal(size=400) * 3, [0.0, 448.0, 500.0, -1000.0, 2.0 ** -9, 2.0 ** -10, 1.0625, 1.1875, 0.0009765625 * 1.5]])
-    tab = e4m3_table()
-    for x in xs.astype(np.float32):
-        assert tab[quantize_e4m3(np.float64(x))] == oracle.round_fp8(float(x), "e4m3"), x
+from _fp8 import e4m3_table, quantize_e4m3
 
 
 @pytest.mark.parametrize("d", [64, 128])
