@@ -94,6 +94,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 {
     using namespace ptx;
     using Cfg = FwdCfg<D>;
+    constexpr bool LEAN = (Cfg::S_BUFS == 1);              // one score buffer: one commit per tile, see the issuer
     extern __shared__ uint8_t smem_raw[];
     uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sQ = smem_u32(sm);                      // also the staging buffer of the O tile
@@ -159,11 +160,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             for (int p = 0; p < Cfg::PANELS; ++p) tma_load_2d(sQ + p * Cfg::Q_PANEL_BYTES, &tmQ, bar(Q_FULL), p * 64, row0);
             for (int j = 0; j < nkv; ++j) {
                 const int s = j % Cfg::STAGES, ph = (j / Cfg::STAGES) & 1;
-                if (!mbar_wait(bar(K_EMPTY + s), ph ^ 1, &abort_flag)) break;
+                if constexpr (LEAN) {                       // K_{j-2} was read by S(j-2), whose commit is S_FULL of that tile
+                    if (j >= 2 && !mbar_wait(bar(S_FULL + (j & 1)), ((j - 2) >> 1) & 1, &abort_flag)) break;
+                } else {
+                    if (!mbar_wait(bar(K_EMPTY + s), ph ^ 1, &abort_flag)) break;
+                }
                 mbar_expect_tx(bar(K_FULL + s), Cfg::KV_BYTES);
                 for (int p = 0; p < Cfg::PANELS; ++p)
                     tma_load_2d(sK0 + s * Cfg::KV_BYTES + p * Cfg::KV_PANEL_BYTES, &tmK, bar(K_FULL + s), p * 64, kvrow0 + j * Cfg::BC);
-                if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1, &abort_flag)) break;
+                if constexpr (LEAN) {                       // V_{j-2} was read by P-bar V of tile j-2, issued before S(j-1): that commit covers it
+                    if (j >= 2 && !mbar_wait(bar(S_FULL + ((j - 1) & 1)), ((j - 1) >> 1) & 1, &abort_flag)) break;
+                } else {
+                    if (!mbar_wait(bar(V_EMPTY + s), ph ^ 1, &abort_flag)) break;
+                }
                 if constexpr (FP8PV) {                      // one box: 64 keys (bytes) x d rows of the transposed V
                     mbar_expect_tx(bar(V_FULL + s), D * Cfg::BC);
                     tma_load_2d(sV0 + s * Cfg::KV_BYTES, &tmV, bar(V_FULL + s), j * Cfg::BC, (bh / prm.group) * D);
@@ -186,9 +195,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const uint64_t dK0 = make_smem_desc(sK0, 16, 1024);
             const uint64_t dV0 = FP8PV ? make_smem_desc_sw64(sV0, 16, 512) : make_smem_desc(sV0, Cfg::KV_PANEL_BYTES, 1024);
             constexpr uint32_t idesc_PV8 = make_idesc_e4m3(128, D);
-            auto issue_S = [&](int j) -> bool {           // S(j) = Q K_j^T
+            // One score buffer (LEAN): the issuer's three waits and four commits per tile sit in the chain
+            // softmax(j) -> P-bar V(j), S(j+1) -> softmax(j+1).  The two waits on TMA barriers are asked ahead of the wait for
+            // P-bar (non-blocking test into a predicate, looked at later; a wait whose answer is used at once costs a
+            // shared-memory round trip), and one commit per tile (after S(j+1)) tells the softmax warps and the producer
+            // everything: it tracks every MMA issued before it.
+            asm volatile(".reg .pred p_kfull, p_vfull;");
+            auto issue_S = [&](int j, bool probed) -> bool {           // S(j) = Q K_j^T
                 const int s = j % Cfg::STAGES, ph = (j / Cfg::STAGES) & 1;
-                if (!mbar_wait(bar(K_FULL + s), ph, &abort_flag)) return false;
+                uint32_t ready = 0;
+                if (LEAN && probed) asm volatile("selp.u32 %0, 1, 0, p_kfull;" : "=r"(ready));
+                if (!ready && !mbar_wait(bar(K_FULL + s), ph, &abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t dK = dK0 + static_cast<uint64_t>((s * Cfg::KV_BYTES) >> 4);
                 const int sb = (Cfg::S_BUFS == 2) ? (j & 1) : 0;
@@ -196,17 +213,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                 for (int k = 0; k < D / 16; ++k)
                     mma_ss(tmem_S + sb * 64, dQ0 + (((k >> 2) * Cfg::Q_PANEL_BYTES + (k & 3) * 32) >> 4),
                            dK + (((k >> 2) * Cfg::KV_PANEL_BYTES + (k & 3) * 32) >> 4), idesc_S, k > 0);
-                mma_commit(bar(S_FULL + sb));
-                mma_commit(bar(K_EMPTY + s));
+                mma_commit(bar(S_FULL + (LEAN ? (j & 1) : sb)));
+                if (!LEAN) mma_commit(bar(K_EMPTY + s));
                 return true;
             };
             bool ok = mbar_wait(bar(Q_FULL), 0, &abort_flag);
-            ok = ok && issue_S(0);
-            if (Cfg::S_BUFS == 2 && nkv > 1) ok = ok && issue_S(1);
+            ok = ok && issue_S(0, false);
+            if (Cfg::S_BUFS == 2 && nkv > 1) ok = ok && issue_S(1, false);
             for (int j = 0; ok && j < nkv; ++j) {
                 const int s = j % Cfg::STAGES, ph = (j / Cfg::STAGES) & 1;
                 const int sb = (Cfg::S_BUFS == 2) ? (j & 1) : 0, sph = (Cfg::S_BUFS == 2) ? ((j >> 1) & 1) : (j & 1);
-                ok = mbar_wait(bar(P_FULL + sb), sph, &abort_flag) && mbar_wait(bar(V_FULL + s), ph, &abort_flag);
+                if constexpr (LEAN) {
+                    asm volatile("mbarrier.test_wait.parity.shared::cta.b64 p_vfull, [%0], %1;"
+                                 ::"r"(bar(V_FULL + s)), "r"(static_cast<uint32_t>(ph)) : "memory");
+                    if (j + 1 < nkv)
+                        asm volatile("mbarrier.test_wait.parity.shared::cta.b64 p_kfull, [%0], %1;"
+                                     ::"r"(bar(K_FULL + (j + 1) % Cfg::STAGES)), "r"(static_cast<uint32_t>(((j + 1) / Cfg::STAGES) & 1)) : "memory");
+                    ok = mbar_wait(bar(P_FULL + sb), sph, &abort_flag);
+                    uint32_t v_ready;
+                    asm volatile("selp.u32 %0, 1, 0, p_vfull;" : "=r"(v_ready));
+                    ok = ok && (v_ready || mbar_wait(bar(V_FULL + s), ph, &abort_flag));
+                } else {
+                    ok = mbar_wait(bar(P_FULL + sb), sph, &abort_flag) && mbar_wait(bar(V_FULL + s), ph, &abort_flag);
+                }
                 if (Cfg::CORR) ok = ok && mbar_wait(bar(O_READY + (j & 1)), (j >> 1) & 1, &abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -223,10 +252,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
                     for (int k = 1; k < Cfg::BC / 16; ++k)
                         mma_ts(tmem_O, tP + k * 8, dV + ((k * 2048) >> 4), idesc_PV, 1u);
                 }
-                mma_commit(pv_done_bar(j));
-                mma_commit(bar(V_EMPTY + s));
+                if constexpr (LEAN) {
+                    if (j == nkv - 1) mma_commit(pv_done_bar(j));      // only the epilogue waits for it
+                } else {
+                    mma_commit(pv_done_bar(j));
+                    mma_commit(bar(V_EMPTY + s));
+                }
                 // the next S for this buffer overwrites it; the MMAs just issued consume its P-bar(j) first
-                if (j + Cfg::S_BUFS < nkv) ok = issue_S(j + Cfg::S_BUFS);
+                if (j + Cfg::S_BUFS < nkv) ok = issue_S(j + Cfg::S_BUFS, true);
             }
         }
         __syncwarp();
@@ -571,8 +604,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         };
 
         for (int j = 0; j < nkv; ++j) {
-            ok = (Cfg::S_BUFS == 2) ? mbar_wait(bar(S_FULL + (j & 1)), (j >> 1) & 1, &abort_flag)
-                                    : mbar_wait(bar(S_FULL), j & 1, &abort_flag);
+            ok = (Cfg::S_BUFS == 2 || LEAN) ? mbar_wait(bar(S_FULL + (j & 1)), (j >> 1) & 1, &abort_flag)
+                                            : mbar_wait(bar(S_FULL), j & 1, &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -583,7 +616,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
         // ---- epilogue: O-bar -> BF16, O = bf16(O-bar / l), L = m + log l
         if (ok) {
-            ok = mbar_wait(pv_done_bar(nkv - 1), pv_done_phase(nkv - 1), &abort_flag);
+            ok = mbar_wait(pv_done_bar(nkv - 1), LEAN ? 0u : pv_done_phase(nkv - 1), &abort_flag);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
