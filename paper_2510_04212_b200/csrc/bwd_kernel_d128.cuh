@@ -300,8 +300,7 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
             }
 #pragma unroll
             for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(sStg_ptr + b * Cfg::PANEL_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) =
-                    make_uint4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
+                sts128(sStg + b * Cfg::PANEL_BYTES + r * 128 + ((c ^ (r & 7)) << 4), x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]);
             fence_proxy_async_smem();
             mbar_arrive(bar(STG_FULL + b));
             ++n;
@@ -362,7 +361,7 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     uint32_t pk[16];
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
-                        const float4 nl = *reinterpret_cast<const float4*>(&sNegL[buf][q0 + c]);
+                        const float4 nl = lds128f(smem_u32(&sNegL[buf][0]) + (q0 + c) * 4);
                         const float nlv[4] = {nl.x, nl.y, nl.z, nl.w};
 #pragma unroll
                         for (int e = 0; e < 4; e += 2) {          // packed FP32 pairs: half the issue slots
@@ -404,7 +403,7 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     uint32_t dsk[8];
 #pragma unroll
                     for (int c = 0; c < 16; c += 4) {
-                        const float4 dl = *reinterpret_cast<const float4*>(&sDelta[buf][q0 + c]);
+                        const float4 dl = lds128f(smem_u32(&sDelta[buf][0]) + (q0 + c) * 4);
                         const float dlv[4] = {dl.x, dl.y, dl.z, dl.w};
                         float ds[4];
 #pragma unroll
@@ -423,8 +422,7 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
 #pragma unroll
                     for (int q2 = 0; q2 < 2; ++q2) {
                         const int cc = h * 2 + q2;
-                        *reinterpret_cast<uint4*>(sX_ptr + half * Cfg::PANEL_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) =
-                            make_uint4(dsk[4 * q2], dsk[4 * q2 + 1], dsk[4 * q2 + 2], dsk[4 * q2 + 3]);
+                        sts128(sX + half * Cfg::PANEL_BYTES + r * 128 + ((cc ^ (r & 7)) << 4), dsk[4 * q2], dsk[4 * q2 + 1], dsk[4 * q2 + 2], dsk[4 * q2 + 3]);
                     }
                 }
             };
@@ -458,7 +456,7 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
                     o.z = pack_bf16(__uint_as_float(a[8 * v + 4]) * mul, __uint_as_float(a[8 * v + 5]) * mul);
                     o.w = pack_bf16(__uint_as_float(a[8 * v + 6]) * mul, __uint_as_float(a[8 * v + 7]) * mul);
                     const int chunk = ((c0 & 63) >> 3) + v;                   // 16-byte chunk inside the 128-byte panel row
-                    *reinterpret_cast<uint4*>(out + (c0 >> 6) * Cfg::PANEL_BYTES + r * 128 + ((chunk ^ (r & 7)) << 4)) = o;
+                    sts128(smem_u32(out) + (c0 >> 6) * Cfg::PANEL_BYTES + r * 128 + ((chunk ^ (r & 7)) << 4), o.x, o.y, o.z, o.w);
                 }
             }
             fence_proxy_async_smem();

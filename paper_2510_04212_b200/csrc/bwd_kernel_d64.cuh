@@ -473,15 +473,13 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int fi = verdict();
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(sStg_ptr + r * 128 + ((c ^ (r & 7)) << 4)) =
-                        make_uint4(a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
+                    sts128(sStg + r * 128 + ((c ^ (r & 7)) << 4), a[4 * c], a[4 * c + 1], a[4 * c + 2], a[4 * c + 3]);
                 panel_written(0);
                 ok = panel_ready(1);
                 if (!ok) break;
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(sStg_ptr + Cfg::TILE_BYTES + r * 128 + ((c ^ (r & 7)) << 4)) =
-                        make_uint4(b[4 * c], b[4 * c + 1], b[4 * c + 2], b[4 * c + 3]);
+                    sts128(sStg + Cfg::TILE_BYTES + r * 128 + ((c ^ (r & 7)) << 4), b[4 * c], b[4 * c + 1], b[4 * c + 2], b[4 * c + 3]);
                 panel_written(1);
                 if (fi >= 0) finish_tile(fi);
             }
@@ -512,7 +510,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         o.z = pack_bf16(__uint_as_float(a[8 * v + 4]) * mul, __uint_as_float(a[8 * v + 5]) * mul);
                         o.w = pack_bf16(__uint_as_float(a[8 * v + 6]) * mul, __uint_as_float(a[8 * v + 7]) * mul);
                         const int cc = (c0 >> 3) + v;
-                        *reinterpret_cast<uint4*>(stage + ((cc ^ (r & 7)) << 4)) = o;
+                        sts128(smem_u32(stage) + ((cc ^ (r & 7)) << 4), o.x, o.y, o.z, o.w);
                     }
                 }
                 if (t == 1) {
@@ -555,7 +553,8 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                uint8_t* xrow = sX_ptr + buf * Cfg::X_BYTES + half * Cfg::TILE_BYTES + r * 128;
+                const uint32_t xrow = sX0 + buf * Cfg::X_BYTES + half * Cfg::TILE_BYTES + r * 128;
+                const uint32_t vecL = smem_u32(&sNegL[buf][0]), vecD = smem_u32(&sDelta[buf][0]);
                 // Partly masked pairs: the causal diagonal (key row r sees query column q only if r <= q), key rows and query
                 // columns beyond the sequence length.  Key row r of the tile sees the query columns q with qlo <= q < qlo + span.
                 // One copy of the arithmetic for both kinds of pair (instruction-cache footprint); the mask sits behind a
@@ -584,8 +583,8 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         uint32_t pk[16], dsk[16];
 #pragma unroll
                         for (int c = 0; c < 32; c += 4) {
-                            const float4 nl = *reinterpret_cast<const float4*>(&sNegL[buf][q0 + c]);
-                            const float4 dl = *reinterpret_cast<const float4*>(&sDelta[buf][q0 + c]);
+                            const float4 nl = lds128f(vecL + (q0 + c) * 4);
+                            const float4 dl = lds128f(vecD + (q0 + c) * 4);
                             const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, dlv[4] = {dl.x, dl.y, dl.z, dl.w};
                             float p[4], ds[4];
 #pragma unroll
@@ -620,8 +619,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
                             const int cc = h * 4 + q4;
-                            *reinterpret_cast<uint4*>(xrow + ((cc ^ (r & 7)) << 4)) =
-                                make_uint4(dsk[4 * q4], dsk[4 * q4 + 1], dsk[4 * q4 + 2], dsk[4 * q4 + 3]);
+                            sts128(xrow + ((cc ^ (r & 7)) << 4), dsk[4 * q4], dsk[4 * q4 + 1], dsk[4 * q4 + 2], dsk[4 * q4 + 3]);
                         }
                     }
                 }

@@ -653,8 +653,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     const int c16 = (c0 >> 3) + v, panel = c16 >> 3, cc = c16 & 7;
-                    *reinterpret_cast<uint4*>(stage + panel * Cfg::Q_PANEL_BYTES + row * 128 + ((cc ^ (row & 7)) << 4)) =
-                        make_uint4(out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
+                    sts128(sQ + panel * Cfg::Q_PANEL_BYTES + row * 128 + ((cc ^ (row & 7)) << 4),
+                           out[4 * v], out[4 * v + 1], out[4 * v + 2], out[4 * v + 3]);
                 }
             }
             prm.lse[static_cast<size_t>(row0) + row] = m + lg2(l) * LN2;

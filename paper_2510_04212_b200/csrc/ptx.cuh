@@ -117,6 +117,18 @@ __device__ __forceinline__ bool mbar_wait_relaxed_ool(uint32_t bar, uint32_t par
     return mbar_try_wait(bar, parity) || mbar_poll_relaxed_ool(bar, parity, abort_flag);
 }
 
+// ---------------------------------------------------------------- shared memory by 32-bit shared address
+// (pointers derived from the aligned dynamic shared-memory base have lost their address space: the compiler would
+// emit generic loads and stores for them)
+__device__ __forceinline__ float4 lds128f(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
