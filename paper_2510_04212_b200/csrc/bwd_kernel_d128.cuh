@@ -79,8 +79,6 @@ attn_bwd_kernel_d128(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t sdO = sQ0 + Cfg::QS * Cfg::TILE_BYTES;
     const uint32_t sX = sdO + Cfg::TILE_BYTES;
     const uint32_t sStg = sX + Cfg::X_BYTES;
-    uint8_t* sX_ptr = sm + (3 + Cfg::QS) * Cfg::TILE_BYTES;
-    uint8_t* sStg_ptr = sX_ptr + Cfg::X_BYTES;
 
     enum { KV_FULL = 0, Q_FULL = 1, Q_EMPTY = 3, DO_FULL = 5, DO_EMPTY = 6, S_FULL = 7, P_FULL = 8, DQ_FULL = 9,
            DQ_EMPTY = 10, DKV_DONE = 11, VEC_FULL = 12, STG_FULL = 14, STG_FREE = 16, DP_FULL = 18, DS_FULL = 19,

@@ -171,8 +171,6 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t sdO0 = sQ0 + Cfg::QS * Cfg::TILE_BYTES;        // QS stages
     const uint32_t sX0 = sdO0 + Cfg::QS * Cfg::TILE_BYTES;        // two buffers
     const uint32_t sStg = sX0 + 2 * Cfg::X_BYTES;                 // two panels of TILE_BYTES
-    uint8_t* sX_ptr = sm + (2 + 2 * Cfg::QS) * Cfg::TILE_BYTES;
-    uint8_t* sStg_ptr = sX_ptr + 2 * Cfg::X_BYTES;
 
     // Barriers.  g = running pair count of this CTA (over all its items), w = running item count, n = running
     // staging step count (one per pair plus one per item).  Unless noted, a barrier completes one phase per g.
@@ -496,7 +494,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (!ok) break;
                 if (t == 0) fi = verdict();
                 const float mul = t ? prm.scale : 1.0f;
-                uint8_t* stage = sStg_ptr + t * Cfg::TILE_BYTES + r * 128;
+                const uint32_t stage = sStg + t * Cfg::TILE_BYTES + r * 128;
 #pragma unroll
                 for (int c0 = 0; c0 < D; c0 += 32) {
                     uint32_t a[32];
@@ -510,7 +508,7 @@ attn_bwd_kernel_d64(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         o.z = pack_bf16(__uint_as_float(a[8 * v + 4]) * mul, __uint_as_float(a[8 * v + 5]) * mul);
                         o.w = pack_bf16(__uint_as_float(a[8 * v + 6]) * mul, __uint_as_float(a[8 * v + 7]) * mul);
                         const int cc = (c0 >> 3) + v;
-                        sts128(smem_u32(stage) + ((cc ^ (r & 7)) << 4), o.x, o.y, o.z, o.w);
+                        sts128(stage + ((cc ^ (r & 7)) << 4), o.x, o.y, o.z, o.w);
                     }
                 }
                 if (t == 1) {

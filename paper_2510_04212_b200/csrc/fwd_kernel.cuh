@@ -623,7 +623,6 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tc_fence_after();
             const float rl = __frcp_rn(l);
             // the Q tile is no longer needed: stage the O tile there in the same swizzled panel layout
-            uint8_t* stage = sm;
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t r[32];
