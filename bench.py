@@ -36,8 +36,8 @@ def flops(B, H, N, d, causal):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_bwd_kernel_d64 launch on C2 (ncu capture summarised in
-# profiles/attn_bwd_kernel_d64_C2.md): 209.3 MB + 111.3 MB.
-BWD_DRAM_BYTES_PER_LAUNCH_C2 = 320.6e6
+# profiles/attn_bwd_kernel_d64_C2.md): 209.9 MB + 111.7 MB.
+BWD_DRAM_BYTES_PER_LAUNCH_C2 = 321.7e6
 
 
 def measured_peaks():
