@@ -322,6 +322,10 @@ def main():
     torch.cuda.set_device(local)
     dist = None
     if world > 1:
+        # NCCL's own log (topology, NVLS, rings) is kept, in a file per rank so that stdout stays the one JSON line;
+        # the only collectives here are the barrier and the MAX over ranks of the timings
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/tmp/nccl_bench_%h_%p.log")
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
